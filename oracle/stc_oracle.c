@@ -1,0 +1,482 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain, slow CPU statement of decode attention over a Quest-selected,
+ * value-group-routed KV cache ("Sub-Token Routing for KV Cache Compression").
+ * It exists so the CUDA library can be checked against something written
+ * straight from the paper.  Only the tests, the smoke check and the
+ * benchmark's CPU-baseline leg may call it.  It shares no code with the CUDA
+ * path and includes no CUDA header.
+ *
+ * Conventions
+ *   - bf16 tensors are passed as uint16_t bit patterns.
+ *   - One "problem" is one (batch, kv head) pair; every function with the
+ *     suffix _batch loops over independent problems (OpenMP static split,
+ *     no other parallelism, no blocking or fusion).
+ *   - head_dim is 128, a page holds 16 tokens.
+ *   - Integer-deciding arithmetic (the page bound) is fp32 in one declared
+ *     summation order; attention arithmetic is fp64.
+ *
+ * Parity status: every function below is pinned by tests/test_oracle_*.py
+ * (closed forms, brute force, textbook attention, invariants).  What is NOT
+ * pinned, because it needs trained weights and evaluation suites: the paper's
+ * accuracy tables -- "parity unpinned" for end-to-end model accuracy.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define D 128
+#define PAGE 16
+
+enum { CLS_DROP = 0, CLS_ROUTED = 1, CLS_FULL = 2 };
+enum { MODE_GLOBAL = 0, MODE_PER_TOKEN = 1 };
+
+static float bf16_to_f32(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* Total order on bf16 bit patterns: numeric order, with -0 below +0. */
+static int32_t bf16_order(uint16_t b) {
+    return (b & 0x8000u) ? -(int32_t)(b & 0x7FFFu) - 1 : (int32_t)b;
+}
+
+/* ------------------------------------------------------------------------
+ * Page metadata: per page and channel, the minimum and maximum key over the
+ * page's valid tokens.  (Quest chunk size 16: Appendix B.1, Table "LLM
+ * training configuration"; the page statistic is Quest's per-channel bound.)
+ * k [len..][128], kmin/kmax [ceil(len/16)][128].
+ * ---------------------------------------------------------------------- */
+void stc_o_page_meta(const uint16_t* k, int32_t len, uint16_t* kmin, uint16_t* kmax) {
+    int32_t n_pages = (len + PAGE - 1) / PAGE;
+    for (int32_t p = 0; p < n_pages; ++p) {
+        for (int c = 0; c < D; ++c) {
+            uint16_t lo = 0, hi = 0;
+            int first = 1;
+            for (int32_t t = p * PAGE; t < (p + 1) * PAGE && t < len; ++t) {
+                uint16_t x = k[(size_t)t * D + c];
+                if (first) { lo = hi = x; first = 0; continue; }
+                if (bf16_order(x) < bf16_order(lo)) lo = x;
+                if (bf16_order(x) > bf16_order(hi)) hi = x;
+            }
+            kmin[(size_t)p * D + c] = lo;
+            kmax[(size_t)p * D + c] = hi;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * Page bound for one query head: U = sum_c max(q_c*kmin_c, q_c*kmax_c), an
+ * upper bound of q.k_t for every token t of the page.
+ *
+ * Declared fp32 summation order (both sides of the parity check must use it,
+ * because the bound decides integers): 16 partial sums; partial l adds the
+ * terms of channels 8l..8l+7 in ascending order starting from +0; the 16
+ * partials are then combined pairwise at distances 8, 4, 2, 1
+ * (s[l] <- s[l] + s[l ^ dist]); the result is s[0].
+ * ---------------------------------------------------------------------- */
+float stc_o_bound_f32(const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax) {
+    float s[16], n[16];
+    for (int l = 0; l < 16; ++l) {
+        float acc = 0.0f;
+        for (int c = 8 * l; c < 8 * l + 8; ++c) {
+            float qc = bf16_to_f32(q[c]);
+            float a = qc * bf16_to_f32(kmin[c]);
+            float b = qc * bf16_to_f32(kmax[c]);
+            float t = a > b ? a : b;
+            acc = acc + t;
+        }
+        s[l] = acc;
+    }
+    for (int dist = 8; dist >= 1; dist >>= 1) {
+        for (int l = 0; l < 16; ++l) n[l] = s[l] + s[l ^ dist];
+        memcpy(s, n, sizeof s);
+    }
+    return s[0];
+}
+
+double stc_o_bound_f64(const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax) {
+    double acc = 0.0;
+    for (int c = 0; c < D; ++c) {
+        double qc = bf16_to_f32(q[c]);
+        double a = qc * bf16_to_f32(kmin[c]);
+        double b = qc * bf16_to_f32(kmax[c]);
+        acc += a > b ? a : b;
+    }
+    return acc;
+}
+
+/* Page scores for one problem: max over the query heads that share the KV
+ * head.  q_group [gq][128]. */
+void stc_o_page_scores(const uint16_t* q_group, int32_t gq, const uint16_t* kmin,
+                       const uint16_t* kmax, int32_t n_pages, float* u) {
+    for (int32_t p = 0; p < n_pages; ++p) {
+        float best = 0.0f;
+        for (int32_t h = 0; h < gq; ++h) {
+            float x = stc_o_bound_f32(q_group + (size_t)h * D, kmin + (size_t)p * D,
+                                      kmax + (size_t)p * D);
+            if (h == 0 || x > best) best = x;
+        }
+        u[p] = best;
+    }
+}
+
+typedef struct { float s; int64_t i; } cand_t;
+
+static int cand_cmp(const void* a, const void* b) {
+    const cand_t* x = (const cand_t*)a;
+    const cand_t* y = (const cand_t*)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    return (x->i > y->i) - (x->i < y->i);   /* ties: lower index first */
+}
+
+static int i32_cmp(const void* a, const void* b) {
+    int32_t x = *(const int32_t*)a, y = *(const int32_t*)b;
+    return (x > y) - (x < y);
+}
+
+/* ------------------------------------------------------------------------
+ * Page selection: keep the k_pg = min(n_pages, budget / 16) pages with the
+ * largest score, ties to the lower page id; ids are emitted ascending.
+ * Returns k_pg.
+ * ---------------------------------------------------------------------- */
+int32_t stc_o_select(const float* u, int32_t n_pages, int32_t token_budget, int32_t* page_ids) {
+    int32_t k_pg = token_budget / PAGE;
+    if (k_pg > n_pages) k_pg = n_pages;
+    if (k_pg < 0) k_pg = 0;
+    cand_t* c = (cand_t*)malloc(sizeof(cand_t) * (size_t)(n_pages > 0 ? n_pages : 1));
+    for (int32_t p = 0; p < n_pages; ++p) { c[p].s = u[p]; c[p].i = p; }
+    qsort(c, (size_t)n_pages, sizeof(cand_t), cand_cmp);
+    for (int32_t j = 0; j < k_pg; ++j) page_ids[j] = (int32_t)c[j].i;
+    qsort(page_ids, (size_t)k_pg, sizeof(int32_t), i32_cmp);
+    free(c);
+    return k_pg;
+}
+
+/* ------------------------------------------------------------------------
+ * Routing mask (Section 3.3 "Routing mask", Section 3.4 global budget,
+ * Appendix B.1 M = N*K).
+ *   scores [len][S]; cls [len] or NULL (all routed); mask [len] out.
+ *   GLOBAL:    N = number of routed tokens, M = N*k_nominal kept pairs.
+ *              min_per_token = 1: each routed token first keeps its best group
+ *              (first maximum), then the best M-N of the remaining pairs are
+ *              kept; min_per_token = 0: the best M of all N*S pairs.
+ *              Ties go to the lower flat index t*S+j.
+ *   PER_TOKEN: every routed token keeps its best k_nominal groups
+ *              (ties to the lower group).
+ *   FULL tokens keep all S groups, DROP tokens none; neither uses budget.
+ * Returns 0, or -1 when M < N with min_per_token = 1, or -2 on bad arguments.
+ * ---------------------------------------------------------------------- */
+int32_t stc_o_route(const float* scores, const uint8_t* cls, int32_t len, int32_t S,
+                    int32_t k_nominal, int32_t min_per_token, int32_t mode, uint16_t* mask) {
+    if (S < 1 || S > 16 || k_nominal < 0 || k_nominal > S) return -2;
+    int64_t n_routed = 0;
+    for (int32_t t = 0; t < len; ++t) {
+        int c = cls ? cls[t] : CLS_ROUTED;
+        mask[t] = (c == CLS_FULL) ? (uint16_t)((1u << S) - 1u) : 0;
+        if (c == CLS_ROUTED) ++n_routed;
+    }
+    if (mode == MODE_PER_TOKEN) {
+        cand_t g[16];
+        for (int32_t t = 0; t < len; ++t) {
+            if ((cls ? cls[t] : CLS_ROUTED) != CLS_ROUTED) continue;
+            for (int j = 0; j < S; ++j) { g[j].s = scores[(size_t)t * S + j]; g[j].i = j; }
+            qsort(g, (size_t)S, sizeof(cand_t), cand_cmp);
+            for (int j = 0; j < k_nominal; ++j) mask[t] |= (uint16_t)(1u << g[j].i);
+        }
+        return 0;
+    }
+    int64_t m_total = n_routed * (int64_t)k_nominal;
+    int64_t take = m_total;
+    if (min_per_token) {
+        if (m_total < n_routed) return -1;
+        take = m_total - n_routed;
+    }
+    cand_t* c = (cand_t*)malloc(sizeof(cand_t) * (size_t)(n_routed * S + 1));
+    int64_t n = 0;
+    for (int32_t t = 0; t < len; ++t) {
+        if ((cls ? cls[t] : CLS_ROUTED) != CLS_ROUTED) continue;
+        int best = -1;
+        if (min_per_token) {
+            best = 0;
+            for (int j = 1; j < S; ++j)
+                if (scores[(size_t)t * S + j] > scores[(size_t)t * S + best]) best = j;
+            mask[t] |= (uint16_t)(1u << best);
+        }
+        for (int j = 0; j < S; ++j) {
+            if (j == best) continue;
+            c[n].s = scores[(size_t)t * S + j];
+            c[n].i = (int64_t)t * S + j;
+            ++n;
+        }
+    }
+    qsort(c, (size_t)n, sizeof(cand_t), cand_cmp);
+    for (int64_t r = 0; r < take && r < n; ++r)
+        mask[c[r].i / S] |= (uint16_t)(1u << (c[r].i % S));
+    free(c);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Packing: walk the tokens in order; offs[t] is the number of groups kept
+ * before token t (offs[len] = total); the kept groups of a token are stored
+ * in ascending group order, each group_dim = 128/S bf16 values.
+ * v [len][128], packed [cap_groups][128/S].  Returns the total, or -1 if it
+ * exceeds cap_groups (nothing past the capacity is written).
+ * ---------------------------------------------------------------------- */
+int64_t stc_o_pack(const uint16_t* v, const uint16_t* mask, int32_t len, int32_t S,
+                   int64_t cap_groups, uint32_t* offs, uint16_t* packed) {
+    int g = D / S;
+    int64_t n = 0;
+    int over = 0;
+    for (int32_t t = 0; t < len; ++t) {
+        offs[t] = (uint32_t)n;
+        for (int j = 0; j < S; ++j) {
+            if (!((mask[t] >> j) & 1u)) continue;
+            if (n < cap_groups)
+                memcpy(packed + (size_t)n * g, v + (size_t)t * D + (size_t)j * g, (size_t)g * 2);
+            else
+                over = 1;
+            ++n;
+        }
+    }
+    offs[len] = (uint32_t)n;
+    return over ? -1 : n;
+}
+
+/* ------------------------------------------------------------------------
+ * Routed attention for one query head (Section 3.3, the attention equation):
+ *   s_t = scale * q.k_t over the tokens of the listed pages (valid tokens
+ *   only), p = softmax(s), out = sum_t p_t * v~_t, where v~_t has the kept
+ *   groups of v_t and zero elsewhere.  The normaliser runs over every listed
+ *   token, whether or not it kept any group.
+ * page_ids NULL = all pages in order.  Values are read from the packed store
+ * through mask/offs.  out [128] fp64; *lse = log sum_t exp(s_t) (natural log).
+ * ---------------------------------------------------------------------- */
+void stc_o_attend_packed(const uint16_t* q, const uint16_t* k, const uint16_t* packed,
+                         const uint16_t* mask, const uint32_t* offs, int32_t len, int32_t S,
+                         const int32_t* page_ids, int32_t n_pages_listed, double scale,
+                         double* out, double* lse) {
+    int g = D / S;
+    int32_t total_pages = (len + PAGE - 1) / PAGE;
+    int32_t n_list = page_ids ? n_pages_listed : total_pages;
+    size_t n_tok = 0;
+    double* s = (double*)malloc(sizeof(double) * ((size_t)n_list * PAGE + 1));
+    int32_t* tok = (int32_t*)malloc(sizeof(int32_t) * ((size_t)n_list * PAGE + 1));
+    for (int32_t i = 0; i < n_list; ++i) {
+        int32_t p = page_ids ? page_ids[i] : i;
+        for (int32_t t = p * PAGE; t < (p + 1) * PAGE && t < len; ++t) {
+            double dot = 0.0;
+            for (int c = 0; c < D; ++c)
+                dot += (double)bf16_to_f32(q[c]) * (double)bf16_to_f32(k[(size_t)t * D + c]);
+            s[n_tok] = dot * scale;
+            tok[n_tok] = t;
+            ++n_tok;
+        }
+    }
+    for (int c = 0; c < D; ++c) out[c] = 0.0;
+    if (n_tok == 0) { if (lse) *lse = -INFINITY; free(s); free(tok); return; }
+    double mx = s[0];
+    for (size_t i = 1; i < n_tok; ++i) if (s[i] > mx) mx = s[i];
+    double den = 0.0;
+    for (size_t i = 0; i < n_tok; ++i) { s[i] = exp(s[i] - mx); den += s[i]; }
+    for (size_t i = 0; i < n_tok; ++i) {
+        int32_t t = tok[i];
+        double p = s[i] / den;
+        int64_t slot = offs[t];
+        for (int j = 0; j < S; ++j) {
+            if (!((mask[t] >> j) & 1u)) continue;
+            for (int e = 0; e < g; ++e)
+                out[j * g + e] += p * (double)bf16_to_f32(packed[(size_t)slot * g + e]);
+            ++slot;
+        }
+    }
+    if (lse) *lse = mx + log(den);
+    free(s);
+    free(tok);
+}
+
+/* Same definition, reading values from the dense V through the mask: the
+ * attention equation applied to v~ = m * v literally. */
+void stc_o_attend_masked_dense(const uint16_t* q, const uint16_t* k, const uint16_t* v,
+                               const uint16_t* mask, int32_t len, int32_t S,
+                               const int32_t* page_ids, int32_t n_pages_listed, double scale,
+                               double* out, double* lse) {
+    int g = D / S;
+    int32_t total_pages = (len + PAGE - 1) / PAGE;
+    int32_t n_list = page_ids ? n_pages_listed : total_pages;
+    size_t n_tok = 0;
+    double* s = (double*)malloc(sizeof(double) * ((size_t)n_list * PAGE + 1));
+    int32_t* tok = (int32_t*)malloc(sizeof(int32_t) * ((size_t)n_list * PAGE + 1));
+    for (int32_t i = 0; i < n_list; ++i) {
+        int32_t p = page_ids ? page_ids[i] : i;
+        for (int32_t t = p * PAGE; t < (p + 1) * PAGE && t < len; ++t) {
+            double dot = 0.0;
+            for (int c = 0; c < D; ++c)
+                dot += (double)bf16_to_f32(q[c]) * (double)bf16_to_f32(k[(size_t)t * D + c]);
+            s[n_tok] = dot * scale;
+            tok[n_tok] = t;
+            ++n_tok;
+        }
+    }
+    for (int c = 0; c < D; ++c) out[c] = 0.0;
+    if (n_tok == 0) { if (lse) *lse = -INFINITY; free(s); free(tok); return; }
+    double mx = s[0];
+    for (size_t i = 1; i < n_tok; ++i) if (s[i] > mx) mx = s[i];
+    double den = 0.0;
+    for (size_t i = 0; i < n_tok; ++i) { s[i] = exp(s[i] - mx); den += s[i]; }
+    for (size_t i = 0; i < n_tok; ++i) {
+        int32_t t = tok[i];
+        double p = s[i] / den;
+        for (int c = 0; c < D; ++c) {
+            double m = (double)((mask[t] >> (c / g)) & 1u);
+            out[c] += p * m * (double)bf16_to_f32(v[(size_t)t * D + c]);
+        }
+    }
+    if (lse) *lse = mx + log(den);
+    free(s);
+    free(tok);
+}
+
+/* Retained-KV fraction by counting stored bytes (Section 3.3 "Compression
+ * ratio", Appendix B.2: rho_total = r * (1 + K/S) / 2): full-width keys of the
+ * retained tokens plus the packed value groups, over dense keys + values of
+ * all original tokens. */
+double stc_o_kv_fraction(int64_t n_tokens_original, int64_t n_tokens_retained,
+                         int64_t n_groups_kept, int32_t S) {
+    double key_bytes = (double)n_tokens_retained * D * 2.0;
+    double val_bytes = (double)n_groups_kept * (D / S) * 2.0;
+    double dense = (double)n_tokens_original * D * 2.0 * 2.0;
+    return (key_bytes + val_bytes) / dense;
+}
+
+/* ========================================================================
+ * Batched drivers over the library's tensor layouts.  Problems (b, kv head)
+ * are independent; the only parallelism is a static split of that loop.
+ *   k, v        [B][Hkv][t_cap][128]
+ *   kmin, kmax  [B][Hkv][p_cap][128],  p_cap = ceil(t_cap/16)
+ *   q           [B][Hq][128]
+ *   scores      [B][Hkv][t_cap][S]
+ *   cls         [B][Hkv or 1][t_cap]   (cls_head_stride = t_cap or 0)
+ *   mask        [B][Hkv][t_cap]; offs [B][Hkv][t_cap+1]
+ *   packed      [B][Hkv][cap_groups][128/S]
+ *   page_ids    [B][Hkv][max_pages]; n_pages [B][Hkv]
+ * seq_len [B] gives the valid tokens per sequence (NULL = t_cap).
+ * ====================================================================== */
+static int32_t len_of(const int32_t* seq_len, int32_t b, int32_t t_cap) {
+    int32_t n = seq_len ? seq_len[b] : t_cap;
+    if (n < 0) n = 0;
+    if (n > t_cap) n = t_cap;
+    return n;
+}
+
+void stc_o_page_meta_batch(int32_t B, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                           const uint16_t* k, uint16_t* kmin, uint16_t* kmax) {
+    int32_t p_cap = (t_cap + PAGE - 1) / PAGE;
+#pragma omp parallel for schedule(static)
+    for (int32_t pr = 0; pr < B * Hkv; ++pr) {
+        int32_t b = pr / Hkv;
+        stc_o_page_meta(k + (size_t)pr * t_cap * D, len_of(seq_len, b, t_cap),
+                        kmin + (size_t)pr * p_cap * D, kmax + (size_t)pr * p_cap * D);
+    }
+}
+
+void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                        const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax,
+                        int32_t token_budget, int32_t max_pages, int32_t* page_ids,
+                        int32_t* n_pages, float* scores_out /* [B][Hkv][p_cap] or NULL */) {
+    int32_t p_cap = (t_cap + PAGE - 1) / PAGE;
+    int32_t gq = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int32_t pr = 0; pr < B * Hkv; ++pr) {
+        int32_t b = pr / Hkv, hk = pr % Hkv;
+        int32_t len = len_of(seq_len, b, t_cap);
+        int32_t np = (len + PAGE - 1) / PAGE;
+        float* u = (float*)malloc(sizeof(float) * (size_t)(p_cap + 1));
+        int32_t* ids = (int32_t*)malloc(sizeof(int32_t) * (size_t)(p_cap + 1));
+        stc_o_page_scores(q + ((size_t)b * Hq + (size_t)hk * gq) * D, gq,
+                          kmin + (size_t)pr * p_cap * D, kmax + (size_t)pr * p_cap * D, np, u);
+        int32_t kp = stc_o_select(u, np, token_budget, ids);
+        if (kp > max_pages) kp = max_pages;   /* caller sized the list too small: truncated */
+        memcpy(page_ids + (size_t)pr * max_pages, ids, sizeof(int32_t) * (size_t)kp);
+        n_pages[pr] = kp;
+        if (scores_out) memcpy(scores_out + (size_t)pr * p_cap, u, sizeof(float) * (size_t)np);
+        free(u);
+        free(ids);
+    }
+}
+
+/* status [B*Hkv]: 0 ok, -1 budget below one group per token, -2 bad args,
+ * -3 capacity overflow.  total [B*Hkv] = groups kept. */
+void stc_o_route_pack_batch(int32_t B, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                            int32_t S, const uint16_t* v, const float* scores,
+                            const uint8_t* cls, int64_t cls_head_stride, int32_t k_nominal,
+                            int32_t min_per_token, int32_t mode, int64_t cap_groups,
+                            uint16_t* mask, uint32_t* offs, uint16_t* packed, int64_t* total,
+                            int32_t* status) {
+    int g = D / S;
+#pragma omp parallel for schedule(static)
+    for (int32_t pr = 0; pr < B * Hkv; ++pr) {
+        int32_t b = pr / Hkv, hk = pr % Hkv;
+        int32_t len = len_of(seq_len, b, t_cap);
+        const uint8_t* c = 0;
+        if (cls) {
+            int64_t per_b = cls_head_stride ? (int64_t)Hkv * cls_head_stride : (int64_t)t_cap;
+            c = cls + (size_t)b * per_b + (size_t)hk * cls_head_stride;
+        }
+        uint16_t* m = mask + (size_t)pr * t_cap;
+        uint32_t* o = offs + (size_t)pr * (t_cap + 1);
+        int32_t rc = stc_o_route(scores + (size_t)pr * t_cap * S, c, len, S, k_nominal,
+                                 min_per_token, mode, m);
+        status[pr] = rc;
+        total[pr] = 0;
+        if (rc != 0) continue;
+        int64_t n = stc_o_pack(v + (size_t)pr * t_cap * D, m, len, S, cap_groups, o,
+                               packed + (size_t)pr * cap_groups * g);
+        if (n < 0) { status[pr] = -3; total[pr] = o[len]; } else total[pr] = n;
+    }
+}
+
+/* use_dense = 0: read values from the packed store; 1: from dense v through
+ * the mask.  out [B][Hq][128] fp64, lse [B][Hq] fp64 (may be NULL). */
+void stc_o_attend_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                        int32_t S, const uint16_t* q, const uint16_t* k, const uint16_t* v_dense,
+                        const uint16_t* packed, int64_t cap_groups, const uint16_t* mask,
+                        const uint32_t* offs, const int32_t* page_ids, const int32_t* n_pages,
+                        int32_t max_pages, double scale, int32_t use_dense, double* out,
+                        double* lse) {
+    int g = D / S;
+    int32_t gq = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int32_t bh = 0; bh < B * Hq; ++bh) {
+        int32_t b = bh / Hq, h = bh % Hq;
+        int32_t pr = b * Hkv + h / gq;
+        int32_t len = len_of(seq_len, b, t_cap);
+        const int32_t* ids = page_ids ? page_ids + (size_t)pr * max_pages : 0;
+        int32_t nl = page_ids ? n_pages[pr] : 0;
+        double* l = lse ? lse + bh : 0;
+        if (use_dense)
+            stc_o_attend_masked_dense(q + (size_t)bh * D, k + (size_t)pr * t_cap * D,
+                                      v_dense + (size_t)pr * t_cap * D, mask + (size_t)pr * t_cap,
+                                      len, S, ids, nl, scale, out + (size_t)bh * D, l);
+        else
+            stc_o_attend_packed(q + (size_t)bh * D, k + (size_t)pr * t_cap * D,
+                                packed + (size_t)pr * cap_groups * g, mask + (size_t)pr * t_cap,
+                                offs + (size_t)pr * (t_cap + 1), len, S, ids, nl, scale,
+                                out + (size_t)bh * D, l);
+    }
+}
+
+int32_t stc_o_max_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
