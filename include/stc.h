@@ -1,0 +1,208 @@
+/*
+ * stc -- decode attention over a two-level compressed KV cache on B200 (sm_100a).
+ *
+ * Level 1 keeps whole tokens: Quest-style page selection scores every 16-token
+ * page of keys by a per-channel min/max bound against the query and keeps the
+ * best pages up to a token budget (the paper's Stage I for LLMs, Section 3.2).
+ * Level 2 keeps parts of tokens: each retained token's value vector is split
+ * into S groups and only the routed groups are stored (Stage II, Section 3.3);
+ * keys stay full width.  Attention is softmax(q K^T / sqrt(d)) V~ with the
+ * dropped groups contributing zero (Section 3.3, attention equation).
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers unless the argument name ends in
+ *     _host.  Tensors are dense, row-major, in the layouts given below.
+ *   - The library is stateless and never allocates or frees device memory;
+ *     scratch space is a caller-provided workspace sized by
+ *     stc_workspace_bytes().  Buffers stay owned by the caller.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*) and
+ *     return without synchronising.
+ *   - Argument errors are detected on the host before anything is enqueued and
+ *     leave every output untouched.  Conditions only the device can see
+ *     (budget too small for the routed-token count, packed-capacity overflow)
+ *     are written to a caller-provided per-problem status array; kernels never
+ *     trap and never read or write out of bounds because of them.
+ *   - head_dim must be 128, page_size 16, n_groups in {4, 8, 16},
+ *     n_q_heads a multiple of n_kv_heads with at most 8 query heads per KV head.
+ *
+ * A "problem" is one (batch, kv head) pair; problems are independent.
+ *
+ * Layouts (B = batch, Hq/Hkv = query / KV heads, T = t_cap, P = ceil(T/16),
+ * S = n_groups, g = 128/S):
+ *   k, v        bf16  [B][Hkv][T][128]
+ *   kmin, kmax  bf16  [B][Hkv][P][128]
+ *   q           bf16  [B][Hq][128]          query head h uses KV head h / (Hq/Hkv)
+ *   scores      f32   [B][Hkv][T][S]        router logits a_{t,j}
+ *   tok_class   u8    [B][Hkv or 1][T]
+ *   v_mask      u16   [B][Hkv][T]           bit j set = group j kept
+ *   v_offs      u32   [B][Hkv][T+1]         groups stored before token t; [len] = total
+ *   v_packed    bf16  [B][Hkv][cap_groups][g]  kept groups, token-major, group-ascending
+ *   page_ids    i32   [B][Hkv][max_pages];  n_pages i32 [B][Hkv]
+ *   out         f32   [B][Hq][128];         lse f32 [B][Hq] (natural log)
+ */
+#ifndef STC_H_
+#define STC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STC_OK = 0,
+    STC_ERR_INVALID_ARG = 1,   /* null pointer, negative size, inconsistent shape      */
+    STC_ERR_UNSUPPORTED = 2,   /* head_dim != 128, page_size != 16, S not in {4,8,16}.. */
+    STC_ERR_WORKSPACE = 3,     /* workspace missing, misaligned (256 B) or too small    */
+    STC_ERR_CAPACITY = 4,      /* packed store too small (device status)                */
+    STC_ERR_BUDGET = 5,        /* fewer kept groups than routed tokens with floor 1     */
+    STC_ERR_CUDA = 6,          /* a CUDA runtime call failed                            */
+    STC_ERR_TIMEOUT = 7        /* reserved: no kernel in this library waits             */
+} stc_status;
+
+enum { STC_CLS_DROP = 0, STC_CLS_ROUTED = 1, STC_CLS_FULL = 2 };
+enum { STC_MODE_GLOBAL = 0, STC_MODE_PER_TOKEN = 1 };
+enum { STC_OP_QUEST_SELECT = 1, STC_OP_ROUTE_PACK = 2, STC_OP_DECODE_ATTN = 3 };
+
+typedef struct stc_shape {
+    int32_t batch, n_q_heads, n_kv_heads;
+    int32_t head_dim;          /* 128 */
+    int32_t page_size;         /* 16  */
+    int32_t n_groups;          /* S   */
+    int32_t t_cap;             /* token capacity = row stride of k, v, scores, v_mask */
+    int32_t reserved;          /* must be 0 */
+    const int32_t* seq_len;    /* device [B] valid tokens per sequence (clamped to
+                                  [0, t_cap] on the device); NULL = t_cap for all    */
+} stc_shape;
+
+typedef struct stc_cache {
+    const void* k;             /* keys, read only                                     */
+    void* kmin;                /* page metadata, written by stc_build_page_meta       */
+    void* kmax;
+    void* v_packed;            /* packed value store, written by stc_route_pack       */
+    uint16_t* v_mask;
+    uint32_t* v_offs;
+    int64_t cap_groups;        /* rows of v_packed per problem                        */
+} stc_cache;
+
+const char* stc_status_string(int32_t status);
+int32_t stc_version(void);
+
+/* Bytes of workspace `op` (STC_OP_*) needs for `shape`; `arg` is max_pages for
+ * STC_OP_DECODE_ATTN and ignored otherwise.  Workspaces must be 256-byte
+ * aligned.  A workspace may be reused by consecutive calls on one stream;
+ * calls that share a workspace must not overlap on the device. */
+int32_t stc_workspace_bytes(const stc_shape* shape, int32_t op, int64_t arg, size_t* bytes_host);
+
+/* Page metadata (Quest chunk size 16: Appendix B.1, "LLM training
+ * configuration"): for pages page_begin <= p < page_end (page_end < 0 = all)
+ * and every channel c,
+ *     kmin[p][c] = min_t k[t][c],  kmax[p][c] = max_t k[t][c]
+ * over the valid tokens t of page p.  Exact (no rounding); -0 orders below
+ * +0.  Pages at or beyond ceil(len/16) are left untouched.
+ * Reads cache->k, writes cache->kmin / kmax. */
+int32_t stc_build_page_meta(const stc_shape* shape, const stc_cache* cache,
+                            int32_t page_begin, int32_t page_end, void* stream);
+
+/* Query-aware page selection (Stage I with Quest, Section 3.2; the paper cites
+ * the criterion, it is stated here): per problem and page
+ *     U[p] = max over the query heads h of the KV head of
+ *            sum_c max(q_h[c]*kmin[p][c], q_h[c]*kmax[p][c])
+ * which bounds q_h.k_t from above for every token of the page (requires
+ * kmin <= kmax as produced by stc_build_page_meta).  The sum is fp32 in a
+ * fixed order: 16 partial sums over channels 8l..8l+7 (ascending, from +0),
+ * combined pairwise at distances 8, 4, 2, 1.  The k_pg = min(ceil(len/16),
+ * token_budget/16) pages with the largest U are kept, ties to the lower page
+ * id; ids are written ascending to page_ids[problem][0..k_pg) and k_pg to
+ * n_pages[problem]; entries past k_pg are left untouched.
+ * max_pages is the row stride of page_ids and must be >=
+ * min(ceil(t_cap/16), token_budget/16).
+ * scores_opt (may be NULL): f32 [B][Hkv][P], receives U for the valid pages.
+ * Non-finite scores are not supported (selection then is unspecified, still
+ * in bounds).  ws: STC_OP_QUEST_SELECT. */
+int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const void* q,
+                         int32_t token_budget, int32_t max_pages, int32_t* page_ids,
+                         int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
+                         void* stream);
+
+/* Sub-token routing and packing (Section 3.3 "Routing mask"; Section 3.4 and
+ * Appendix B.1 for the global budget M = N*K; the VLM per-token rule is the
+ * fixed top-K of Section 3.5 / Appendix B.1).
+ *   tok_class (NULL = every valid token ROUTED): DROP tokens store nothing,
+ *   FULL tokens store all S groups, neither uses budget.  class_head_stride
+ *   is T when classes differ per KV head and 0 when one [B][T] array serves
+ *   all heads.
+ *   STC_MODE_GLOBAL: with N routed tokens in the problem, M = N*k_nominal
+ *   (token, group) pairs are kept.  min_per_token = 1: each routed token
+ *   keeps its highest-scoring group (first maximum), then the M-N best of the
+ *   remaining pairs are kept; min_per_token = 0: the M best of all pairs
+ *   (tokens may end with no group, as in the paper's Fig. 1).  Ties go to
+ *   the lower flat index t*S + j; -0 and +0 compare equal.
+ *   STC_MODE_PER_TOKEN: every routed token keeps its k_nominal best groups
+ *   (ties to the lower group).
+ * Outputs: out->v_mask (0 for tokens past len), out->v_offs[0..len],
+ * out->v_packed, total_groups i64 [B][Hkv], status i32 [B][Hkv] (STC_OK,
+ * STC_ERR_BUDGET: nothing packed for that problem, or STC_ERR_CAPACITY: groups
+ * past cap_groups were not stored).  Non-finite scores are not supported.
+ * ws: STC_OP_ROUTE_PACK. */
+int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* scores,
+                       const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
+                       int32_t min_per_token, int32_t mode, const stc_cache* out,
+                       int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes,
+                       void* stream);
+
+/* Routed decode attention (Section 3.3, attention equation): per query head h
+ * with KV head h / (Hq/Hkv) and R = the valid tokens of the listed pages,
+ *     s_t = sm_scale * q_h.k_t,  p = softmax over R of s,
+ *     out[h][j*g .. (j+1)*g) = sum_{t in R} p_t * [bit j of v_mask[t]] * v_t^{(j)}
+ * so a dropped group adds zero while its token still counts in the
+ * normaliser.  page_ids NULL = every page of the sequence (selection off);
+ * otherwise n_pages[problem] ids are read from page_ids[problem] (row stride
+ * max_pages); ids outside [0, ceil(len/16)) are skipped, a page listed twice
+ * counts twice.  An empty R gives out = 0 and lse = -inf.
+ * bf16 inputs, fp32 accumulation, fp32 outputs; the softmax weights enter the
+ * value contraction as a bf16 pair (high + residual part) when the tensor-core
+ * path is used (more than one query head per KV head).  lse_opt may be NULL.
+ * ws: STC_OP_DECODE_ATTN with arg = max_pages (for page_ids NULL: ceil(T/16)). */
+int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const void* q,
+                        const int32_t* page_ids, const int32_t* n_pages, int32_t max_pages,
+                        float sm_scale, float* out, float* lse_opt, void* ws, size_t ws_bytes,
+                        void* stream);
+
+/* Stored bytes of the compressed cache for the accounting of Section 3.3
+ * ("Compression ratio") and Appendix B.2: full-width keys of the retained
+ * tokens plus the packed groups (mask/offset/metadata bytes are returned
+ * separately).  Host arithmetic only. */
+int32_t stc_cache_bytes(int64_t n_tokens_retained, int64_t n_groups_kept, int32_t n_groups,
+                        int64_t* kv_bytes_host, int64_t* index_bytes_host);
+
+/* One whole pass from HOST memory (the end-to-end form of the calls above):
+ * copies k, v, scores, tok_class and q from host buffers into a caller-provided
+ * device arena, runs stc_build_page_meta, stc_route_pack (STC_MODE_* / floor as
+ * given), stc_quest_select (skipped when token_budget < 0: every page attended)
+ * and stc_decode_attn, and copies out [B][Hq][128], total_groups [B][Hkv] and
+ * status [B][Hkv] back to host buffers.  Everything is enqueued on `stream`;
+ * the host outputs are valid after the caller synchronises the stream.  Host
+ * buffers should be page-locked so the copies run asynchronously.
+ *   *_host       host pointers, same layouts as the device tensors;
+ *                tok_class_host is [B][T] shared by heads, or NULL
+ *   shape->seq_len  still a DEVICE pointer (or NULL)
+ *   cap_groups   rows of the packed store per problem inside the arena
+ *   arena        device memory, 256-byte aligned, at least
+ *                stc_pass_host_arena_bytes() bytes; owned by the caller and
+ *                reusable by the next call on the same stream
+ * Operation and errors are those of the four calls it chains. */
+int32_t stc_pass_host_arena_bytes(const stc_shape* shape, int64_t cap_groups, int32_t token_budget,
+                                  size_t* bytes_host);
+int32_t stc_pass_host(const stc_shape* shape, const void* k_host, const void* v_host,
+                      const float* scores_host, const uint8_t* tok_class_host, const void* q_host,
+                      int32_t token_budget, int32_t k_nominal, int32_t min_per_token, int32_t mode,
+                      float sm_scale, int64_t cap_groups, void* arena, size_t arena_bytes,
+                      float* out_host, int64_t* total_groups_host, int32_t* status_host,
+                      void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STC_H_ */

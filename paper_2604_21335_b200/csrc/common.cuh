@@ -1,0 +1,71 @@
+// Shared device helpers and internal launch declarations for libstc (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "stc.h"
+
+namespace stc {
+
+constexpr int kHeadDim = 128;
+constexpr int kPage = 16;
+constexpr int kRowBytes = kHeadDim * 2;        // one key / value row
+constexpr int kOctets = kHeadDim / 8;          // 16-byte chunks per row
+
+// Geometry resolved once on the host.
+struct Geom {
+    int B, Hq, Hkv, Gq, S, g, T, P;            // P = ceil(T/16)
+    int problems;
+    const int32_t* seq_len;
+};
+
+__device__ __forceinline__ int clamp_len(const int32_t* seq_len, int b, int T) {
+    int n = seq_len ? seq_len[b] : T;
+    return n < 0 ? 0 : (n > T ? T : n);
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint4 ldg_nc16(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// Order-preserving map from fp32 bits to uint32 (larger float -> larger key);
+// -0 is folded onto +0 so the two compare equal.
+__device__ __forceinline__ uint32_t float_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    if ((u << 1) == 0u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// ---- internal launchers (one per source file) -------------------------------
+cudaError_t launch_page_meta(const Geom& g, const void* k, void* kmin, void* kmax, int page_begin,
+                             int page_end, cudaStream_t st);
+
+size_t select_ws_bytes(const Geom& g);
+cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
+                                int token_budget, int max_pages, int32_t* page_ids,
+                                int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st);
+
+size_t route_ws_bytes(const Geom& g);
+cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
+                              const uint8_t* tok_class, int64_t class_head_stride, int k_nominal,
+                              int min_per_token, int mode, void* v_packed, uint16_t* v_mask,
+                              uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups,
+                              int32_t* status, void* ws, cudaStream_t st);
+
+struct AttnPlan { int pages_per_cta, n_splits; };
+AttnPlan attn_plan(const Geom& g, int max_pages);
+size_t attn_ws_bytes(const Geom& g, int max_pages);
+cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packed,
+                               const uint16_t* v_mask, const uint32_t* v_offs, int64_t cap_groups,
+                               const void* q, const int32_t* page_ids, const int32_t* n_pages,
+                               int max_pages, float sm_scale, float* out, float* lse, void* ws,
+                               cudaStream_t st);
+
+}  // namespace stc

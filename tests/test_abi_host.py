@@ -1,0 +1,96 @@
+"""Host-only checks of the C-ABI library: it loads, exports every symbol the
+header declares, and rejects bad arguments before touching the device."""
+import ctypes as C
+import re
+from pathlib import Path
+
+import pytest
+
+import paper_2604_21335_b200 as P
+from paper_2604_21335_b200 import binding as Bd
+from paper_2604_21335_b200 import build as B
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build()
+    return P.load_library()
+
+
+def declared_symbols():
+    names = set()
+    for h in (ROOT / "include").glob("*.h"):
+        names |= set(re.findall(r"\b(stc_[a-z_0-9]+)\s*\(", h.read_text()))
+    return names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_symbols()
+    assert set(Bd.EXPORTS) <= names and len(names) >= 8
+    for n in names:
+        assert hasattr(lib, n), n
+    assert lib.stc_version() >= 100
+    assert lib.stc_status_string(0) == b"ok"
+    assert b"workspace" in lib.stc_status_string(3)
+
+
+def shape(**kw):
+    base = dict(batch=1, n_q_heads=8, n_kv_heads=8, n_groups=8, t_cap=4096)
+    base.update(kw)
+    return P.Shape(**base)
+
+
+def test_workspace_sizes_and_shape_validation(lib):
+    s = shape()
+    for op in (Bd.OP_QUEST_SELECT, Bd.OP_ROUTE_PACK, Bd.OP_DECODE_ATTN):
+        n = P.workspace_bytes(s, op, 64)
+        assert n > 0 and n % 256 == 0
+    assert P.workspace_bytes(shape(batch=0), Bd.OP_ROUTE_PACK) == 0
+    for bad, code in [(dict(head_dim=64), 2), (dict(page_size=32), 2), (dict(n_groups=5), 2),
+                      (dict(n_q_heads=9), 1), (dict(n_q_heads=72), 2), (dict(t_cap=-1), 1),
+                      (dict(t_cap=1 << 28), 2)]:
+        with pytest.raises(P.StcError) as e:
+            P.workspace_bytes(shape(**bad), Bd.OP_QUEST_SELECT)
+        assert e.value.code == code, bad
+    with pytest.raises(P.StcError):
+        P.workspace_bytes(s, 99)
+
+
+def test_calls_reject_bad_arguments_before_any_launch(lib):
+    cs = shape().c()
+    cc = Bd._Cache()                      # all null
+    st = None
+    assert lib.stc_build_page_meta(C.byref(cs), C.byref(cc), 0, -1, st) == 1
+    assert lib.stc_build_page_meta(None, C.byref(cc), 0, -1, st) == 1
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), None, 1024, 64, None, None, None, None, 0, st) == 1
+    assert lib.stc_route_pack(C.byref(cs), None, None, None, 0, 4, 1, 0, C.byref(cc), None, None, None, 0, st) == 1
+    assert lib.stc_route_pack(C.byref(cs), None, None, None, 0, 9, 1, 0, C.byref(cc), None, None, None, 0, st) == 1
+    assert lib.stc_route_pack(C.byref(cs), None, None, None, 17, 4, 1, 0, C.byref(cc), None, None, None, 0, st) == 1
+    assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), None, None, None, 0, 0.1, None, None, None, 0, st) == 1
+    # non-null fakes (never dereferenced on the host) reach the workspace checks
+    fake = C.c_void_p(0x1000)
+    cc = Bd._Cache(fake, fake, fake, fake, fake, fake, 100)
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 63, fake, fake, None, fake, 1 << 30, st) == 1
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, None, None, 0, st) == 3
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, None, C.c_void_p(0x1010), 1 << 30, st) == 3
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, None, fake, 16, st) == 3
+    assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, None, 64, 0.1, fake, None, fake, 1 << 30, st) == 1
+    assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, fake, 64, 0.1, fake, None, fake, 16, st) == 3
+
+
+def test_cache_bytes_reproduces_the_closed_form(lib):
+    # r = 1/4 of 2048 tokens, K/S = 2/8: (512*256 + 1024*32) / (2048*512) = 15.625 %
+    kv, idx = P.cache_bytes(512, 1024, 8)
+    assert kv / (2048 * 512) == 0.15625
+    assert idx == 512 * 2 + 513 * 4 + 32 * 512
+    kv, _ = P.cache_bytes(256, 256 * 7, 8)                 # r = 1/8, K/S = 7/8
+    assert kv / (2048 * 512) == 0.1171875
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(Bd, "_lib", None)
+    monkeypatch.setattr(Bd, "_LIB_PATH", tmp_path / "libstc.so")
+    with pytest.raises(ImportError):
+        Bd.load_library()

@@ -1,0 +1,228 @@
+"""Parity of the CUDA path (through the C-ABI binding) against the CPU checker.
+
+Integer and byte results (page metadata, page ids, masks, offsets, packed
+store) must be bit-exact; attention outputs must be within max-abs 1e-2 and
+mean relative error 2e-3 of the fp64 checker."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2604_21335_b200 as P
+from paper_2604_21335_b200 import binding as Bd
+from paper_2604_21335_b200 import workload as W
+
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def full_parity(w, seq_len=None, **kw):
+    d = W.make_inputs(w, DEV)
+    g = H.gpu_pipeline(w, d, seq_len=seq_len, **kw)
+    o = H.oracle_pipeline(w, d, seq_len=seq_len, **{k: v for k, v in kw.items() if k != "want_scores"})
+    H.assert_bit_exact_write_side(w, g, o)
+    if o["page_ids"] is not None:
+        H.assert_bit_exact_selection(g, o)
+    errs = H.assert_attention_close(g, o)
+    return d, g, o, errs
+
+
+def test_cfg0_tiny_mha_full():
+    w = W.get("cfg0")
+    d, g, o, errs = full_parity(w)
+    assert (o["n_pages"] == 64).all()
+    assert (o["total"] == 4096 * 4).all()                 # M = N*K exactly
+    cnt = np.vectorize(lambda x: bin(int(x)).count("1"))(o["mask"])
+    assert cnt.min() >= 1
+
+
+SHRUNK = [
+    # name, overrides, seq_len (ragged) -- several tiles, ragged tails
+    ("cfg1", dict(n_q_heads=4, n_kv_heads=4, t_cache=16 * 150 + 7, token_budget=16 * 21), None),
+    ("cfg1", dict(n_q_heads=3, n_kv_heads=3, batch=2, t_cache=2500, token_budget=512), [2500, 1031]),
+    ("cfg2", dict(batch=2, t_cache=16 * 140 + 3, token_budget=16 * 40), [16 * 140 + 3, 1777]),
+    ("cfg2", dict(batch=1, n_q_heads=8, n_kv_heads=2, t_cache=3000, token_budget=16 * 9), None),   # Gq = 4, S = 16
+    ("cfg4", dict(batch=2, n_q_heads=8, n_kv_heads=2, t_cache=16 * 300 + 1, token_budget=1024), [4801, 16 * 77]),
+    ("cfg4", dict(batch=1, n_q_heads=16, n_kv_heads=2, t_cache=2100, token_budget=256, k_nominal=2), None),  # Gq = 8
+    ("cfg4", dict(batch=1, n_q_heads=10, n_kv_heads=2, t_cache=1500, token_budget=160, n_groups=4, k_nominal=1), None),  # Gq=5,S=4
+    ("cfg3", dict(batch=3, n_q_heads=4, n_kv_heads=4), None),
+]
+
+
+@pytest.mark.parametrize("name,over,seq", SHRUNK)
+def test_shrunken_configs(name, over, seq):
+    w = W.shrink(W.get(name), **over)
+    full_parity(w, seq_len=seq)
+
+
+def test_cfg3_class_layout_and_totals():
+    w = W.shrink(W.get("cfg3"), batch=2, n_q_heads=8, n_kv_heads=8)
+    d, g, o, _ = full_parity(w)
+    assert w.t_cache == 272 and o["page_ids"] is None
+    assert (o["total"] == 128 * 8 + 144 * 3).all()        # full text tokens + M = 144*3
+    assert (o["mask"][:, :, :128] == 0xFF).all()
+
+
+def test_budget_covers_everything_and_all_groups_equals_dense_attention():
+    w = W.shrink(W.get("cfg0"), n_q_heads=4, n_kv_heads=4, t_cache=16 * 40 + 9, token_budget=16 * 64,
+                 k_nominal=8)
+    d, g, o, _ = full_parity(w)
+    ids = g["page_ids"].cpu().numpy()
+    assert (g["n_pages"].cpu().numpy() == 41).all()
+    assert (ids[:, :, :41] == np.arange(41)).all()
+    # all pages + all groups: textbook dense softmax attention (library routine, fp32 inputs)
+    q = d["q"][0].float().cpu()[0][:, None, :]           # [H,1,128]
+    ref = torch.nn.functional.scaled_dot_product_attention(q.double(), d["k"][0].cpu().double(),
+                                                           d["v"][0].cpu().double())[:, 0]
+    err = (g["out"][0].cpu().double() - ref).abs().max().item()
+    assert err < 1e-2
+
+
+@pytest.mark.parametrize("kn,mpt,mode", [(1, 1, 0), (8, 1, 0), (2, 0, 0), (7, 1, 0), (2, 1, 1), (3, 1, 1)])
+def test_routing_modes(kn, mpt, mode):
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=2309, token_budget=320, k_nominal=kn)
+    full_parity(w, min_per_token=mpt, mode=mode)
+
+
+def test_injected_ties_resolve_to_lower_indices():
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=16 * 64, token_budget=16 * 10)
+    d = W.make_inputs(w, DEV)
+    # duplicate page contents -> exact ties between page bounds
+    k = d["k"].view(1, 2, 64, 16, 128)
+    k[:, :, 1::2] = k[:, :, 0::2].clone()
+    # quantised router scores -> massive ties at the routing threshold
+    d["scores"] = torch.round(d["scores"] * 2) / 2
+    d["scores"][0, 0, 100:200] = 0.0
+    d["scores"][0, 1, :, :] = -0.0
+    g = H.gpu_pipeline(w, d)
+    o = H.oracle_pipeline(w, d)
+    H.assert_bit_exact_write_side(w, g, o)
+    H.assert_bit_exact_selection(g, o)
+    H.assert_attention_close(g, o)
+    u = o["u"][0, 0]
+    assert H.near_tie_pages(u, 10) >= 1                   # the duplicated pages do tie
+
+
+def test_page_meta_signed_zero_and_partial_page():
+    w = W.shrink(W.get("cfg0"), n_q_heads=1, n_kv_heads=1, t_cache=40, token_budget=32)
+    d = W.make_inputs(w, DEV)
+    kb = d["k"].view(torch.int16)
+    kb[0, 0, 0, :] = -32768      # -0.0
+    kb[0, 0, 1, :] = 0           # +0.0
+    kb[0, 0, 2:16, :] = 0
+    g = H.gpu_pipeline(w, d, seq_len=[35])
+    o = H.oracle_pipeline(w, d, seq_len=[35])
+    H.assert_bit_exact_write_side(w, g, o)
+    assert (H.np_u16(g["cache"].kmin)[0, 0, 0] == 0x8000).all()
+    assert (H.np_u16(g["cache"].kmax)[0, 0, 0] == 0x0000).all()
+
+
+def test_empty_and_single_token_sequences():
+    w = W.shrink(W.get("cfg2"), batch=3, t_cache=200, token_budget=64)
+    d = W.make_inputs(w, DEV)
+    seq = [0, 1, 200]
+    g = H.gpu_pipeline(w, d, seq_len=seq)
+    o = H.oracle_pipeline(w, d, seq_len=seq)
+    H.assert_bit_exact_write_side(w, g, o)
+    H.assert_bit_exact_selection(g, o)
+    H.assert_attention_close(g, o)
+    assert (g["out"][0] == 0).all() and torch.isinf(g["lse"][0]).all()
+
+
+def test_zero_token_budget_selects_nothing():
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=300)
+    d = W.make_inputs(w, DEV)
+    g = H.gpu_pipeline(w, d, budget=15)
+    assert (g["n_pages"] == 0).all() and (g["out"] == 0).all()
+
+
+def test_device_status_budget_and_capacity():
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=1000, token_budget=160)
+    d = W.make_inputs(w, DEV)
+    g = H.gpu_pipeline(w, d, k_nominal=0, min_per_token=1)           # M < N
+    assert (g["status"] == 5).all() and (g["total"] == 0).all()
+    assert (g["cache"].v_mask == 0).all()
+    cap = 1000 * 4 - 100
+    g = H.gpu_pipeline(w, d, cap_groups=cap)                         # store too small: no overflow writes
+    o = H.oracle_pipeline(w, d, cap_groups=cap)
+    assert (g["status"] == 4).all() and (o["status"] == -3).all()
+    np.testing.assert_array_equal(g["total"].cpu().numpy(), o["total"])
+    np.testing.assert_array_equal(H.np_u16(g["cache"].v_packed), o["packed"])
+
+
+def test_out_of_range_and_repeated_page_ids():
+    w = W.shrink(W.get("cfg2"), batch=1, t_cache=16 * 20 + 5, token_budget=None)
+    d = W.make_inputs(w, DEV)
+    ids = torch.tensor([[3, 3, -1, 99, 20, 0, 7, 7]], dtype=torch.int32, device=DEV).repeat(4, 1)[None]
+    n = torch.tensor([[8, 6, 0, 3]], dtype=torch.int32, device=DEV)
+    g = H.gpu_pipeline(w, d, page_ids_override=(ids.contiguous(), n))
+    valid = [[p for p in row[:k] if 0 <= p < 21] for row, k in zip(ids[0].tolist(), n[0].tolist())]
+    width = max(1, max(len(v) for v in valid))
+    ids_o = np.zeros((1, 4, width), np.int32); n_o = np.zeros((1, 4), np.int32)
+    for h, v in enumerate(valid):
+        ids_o[0, h, :len(v)] = v; n_o[0, h] = len(v)
+    o = H.oracle_pipeline(w, d, page_ids_override=(ids_o, n_o))
+    H.assert_attention_close(g, o)
+
+
+def test_selection_is_deterministic_and_workspace_reusable():
+    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=8, n_kv_heads=2, t_cache=16 * 700, token_budget=1024)
+    d = W.make_inputs(w, DEV, n_queries=3)
+    a = H.gpu_pipeline(w, d, q_index=1)
+    b = H.gpu_pipeline(w, d, q_index=1)
+    assert torch.equal(a["page_ids"], b["page_ids"]) and torch.equal(a["cache"].v_mask, b["cache"].v_mask)
+    assert torch.equal(a["cache"].v_offs, b["cache"].v_offs)
+    # attention merges split-K partials in a fixed order: bitwise repeatable
+    assert torch.equal(a["out"], b["out"])
+    o = H.oracle_pipeline(w, d, q_index=1)
+    H.assert_bit_exact_selection(a, o)
+
+
+def _problem_slice(w, d, b, hk):
+    """One (batch, kv head) problem as a standalone B=1, Hkv=1 workload on the CPU."""
+    gq = w.gq
+    w1 = W.shrink(w, batch=1, n_q_heads=gq, n_kv_heads=1)
+    d1 = dict(k=d["k"][b:b + 1, hk:hk + 1].cpu(), v=d["v"][b:b + 1, hk:hk + 1].cpu(),
+              q=d["q"][:, b:b + 1, hk * gq:(hk + 1) * gq].cpu(),
+              scores=d["scores"][b:b + 1, hk:hk + 1].cpu(),
+              tok_class=None if d["tok_class"] is None else d["tok_class"][b:b + 1].cpu(),
+              seq_len=d["seq_len"][b:b + 1].cpu())
+    return w1, d1
+
+
+@pytest.mark.parametrize("name,samples", [("cfg1", [(0, 0), (0, 13), (0, 31)]),
+                                          ("cfg2", [(0, 0), (5, 2), (7, 3)])])
+def test_full_size_sampled_problems(name, samples):
+    """At the benchmarked sizes: whole pass on the GPU, sampled problems on the checker."""
+    w = W.get(name)
+    d = W.make_inputs(w, DEV)
+    g = H.gpu_pipeline(w, d)
+    S = w.n_groups
+    # properties that hold at any size
+    cnt = torch.zeros_like(g["cache"].v_mask, dtype=torch.int32)
+    for j in range(S):
+        cnt += (g["cache"].v_mask.int() >> j) & 1
+    assert (cnt.sum(-1) == w.t_cache * w.k_nominal).all() and cnt.min() >= 1
+    assert (g["total"] == w.t_cache * w.k_nominal).all() and (g["status"] == 0).all()
+    offs = g["cache"].v_offs.long()
+    assert torch.equal(offs[..., 1:] - offs[..., :-1], cnt.long())
+    ids = g["page_ids"]
+    assert (ids[..., 1:] > ids[..., :-1]).all() and (g["n_pages"] == w.token_budget // 16).all()
+    for b, hk in samples:
+        w1, d1 = _problem_slice(w, d, b, hk)
+        o = H.oracle_pipeline(w1, d1)
+        g1 = dict(cache=P.Cache(kmin=g["cache"].kmin[b:b + 1, hk:hk + 1].contiguous(),
+                                kmax=g["cache"].kmax[b:b + 1, hk:hk + 1].contiguous(),
+                                v_mask=g["cache"].v_mask[b:b + 1, hk:hk + 1].contiguous(),
+                                v_offs=g["cache"].v_offs[b:b + 1, hk:hk + 1].contiguous(),
+                                v_packed=g["cache"].v_packed[b:b + 1, hk:hk + 1].contiguous()),
+                  total=g["total"][b:b + 1, hk:hk + 1], status=g["status"][b:b + 1, hk:hk + 1],
+                  page_ids=g["page_ids"][b:b + 1, hk:hk + 1], n_pages=g["n_pages"][b:b + 1, hk:hk + 1],
+                  u=g["u"][b:b + 1, hk:hk + 1],
+                  out=g["out"][b:b + 1, hk * w.gq:(hk + 1) * w.gq],
+                  lse=g["lse"][b:b + 1, hk * w.gq:(hk + 1) * w.gq])
+        H.assert_bit_exact_write_side(w1, g1, o)
+        H.assert_bit_exact_selection(g1, o)
+        H.assert_attention_close(g1, o)
