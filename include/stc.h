@@ -111,8 +111,9 @@ int32_t stc_build_page_meta(const stc_shape* shape, const stc_cache* cache,
  *            sum_c max(q_h[c]*kmin[p][c], q_h[c]*kmax[p][c])
  * which bounds q_h.k_t from above for every token of the page (requires
  * kmin <= kmax as produced by stc_build_page_meta).  The sum is fp32 in a
- * fixed order: 16 partial sums over channels 8l..8l+7 (ascending, from +0),
- * combined pairwise at distances 8, 4, 2, 1.  The k_pg = min(ceil(len/16),
+ * fixed order: 16 partial sums, partial l = (sum of the even channels of
+ * 8l..8l+7, ascending, from +0) + (the same over the odd channels); the
+ * partials are combined pairwise at distances 8, 4, 2, 1.  The k_pg = min(ceil(len/16),
  * token_budget/16) pages with the largest U are kept, ties to the lower page
  * id; ids are written ascending to page_ids[problem][0..k_pg) and k_pg to
  * n_pages[problem]; entries past k_pg are left untouched.

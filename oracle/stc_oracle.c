@@ -74,23 +74,25 @@ void stc_o_page_meta(const uint16_t* k, int32_t len, uint16_t* kmin, uint16_t* k
  * upper bound of q.k_t for every token t of the page.
  *
  * Declared fp32 summation order (both sides of the parity check must use it,
- * because the bound decides integers): 16 partial sums; partial l adds the
- * terms of channels 8l..8l+7 in ascending order starting from +0; the 16
- * partials are then combined pairwise at distances 8, 4, 2, 1
- * (s[l] <- s[l] + s[l ^ dist]); the result is s[0].
+ * because the bound decides integers): 16 partial sums; partial l covers
+ * channels 8l..8l+7 and is formed as even + odd, where even adds the terms of
+ * channels 8l, 8l+2, 8l+4, 8l+6 in ascending order starting from +0 and odd
+ * does the same for 8l+1, 8l+3, 8l+5, 8l+7; the 16 partials are then combined
+ * pairwise at distances 8, 4, 2, 1 (s[l] <- s[l] + s[l ^ dist]); the result
+ * is s[0].
  * ---------------------------------------------------------------------- */
 float stc_o_bound_f32(const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax) {
     float s[16], n[16];
     for (int l = 0; l < 16; ++l) {
-        float acc = 0.0f;
+        float part[2] = {0.0f, 0.0f};           /* [0] even channels, [1] odd channels */
         for (int c = 8 * l; c < 8 * l + 8; ++c) {
             float qc = bf16_to_f32(q[c]);
             float a = qc * bf16_to_f32(kmin[c]);
             float b = qc * bf16_to_f32(kmax[c]);
             float t = a > b ? a : b;
-            acc = acc + t;
+            part[c & 1] = part[c & 1] + t;
         }
-        s[l] = acc;
+        s[l] = part[0] + part[1];
     }
     for (int dist = 8; dist >= 1; dist >>= 1) {
         for (int l = 0; l < 16; ++l) n[l] = s[l] + s[l ^ dist];

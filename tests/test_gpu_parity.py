@@ -131,6 +131,16 @@ def test_empty_and_single_token_sequences():
     assert (g["out"][0] == 0).all() and torch.isinf(g["lse"][0]).all()
 
 
+def test_more_pages_than_the_register_topk_holds():
+    # > 8192 pages per problem takes the memory-resident top-k path
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=1, t_cache=16 * 8300 + 5, token_budget=16 * 300)
+    d = W.make_inputs(w, DEV)
+    g = H.gpu_pipeline(w, d)
+    o = H.oracle_pipeline(w, d)
+    H.assert_bit_exact_selection(g, o)
+    H.assert_attention_close(g, o)
+
+
 def test_zero_token_budget_selects_nothing():
     w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=300)
     d = W.make_inputs(w, DEV)

@@ -118,12 +118,22 @@ def test_bound_summation_order_hand_cases():
     t = [0.0] * 128
     t[0] = big; t[8] = 1.0; t[64] = -big
     assert _bound_with_terms(t) == 1.0
-    # (c) inside a partial the channels are added left to right:
-    #     (2^24 + 1) rounds to 2^24, then -2^24 gives 0 (not 1).
+    # (c) inside a partial, even and odd channels are summed separately:
+    #     even = 2^24 - 2^24 = 0, odd = 1, partial = 1 (one running sum over all
+    #     eight channels would round 2^24 + 1 to 2^24 and give 0).
     t = [0.0] * 128
     t[0] = big; t[1] = 1.0; t[2] = -big
+    assert _bound_with_terms(t) == 1.0
+    # (d) each of the two running sums goes left to right: (2^24 + 1) rounds to
+    #     2^24 before -2^24 arrives, so the one is lost, on the even side ...
+    t = [0.0] * 128
+    t[0] = big; t[2] = 1.0; t[4] = -big
     assert _bound_with_terms(t) == 0.0
-    # (d) partials are 8 channels wide: channel 8 starts a new partial, so the
+    #     ... and on the odd side.
+    t = [0.0] * 128
+    t[1] = big; t[3] = 1.0; t[7] = -big
+    assert _bound_with_terms(t) == 0.0
+    # (e) partials are 8 channels wide: channel 8 starts a new partial, so the
     #     one survives there.
     t = [0.0] * 128
     t[7] = big; t[8] = 1.0; t[71] = -big
