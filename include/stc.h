@@ -58,7 +58,8 @@ typedef enum {
     STC_ERR_CAPACITY = 4,      /* packed store too small (device status)                */
     STC_ERR_BUDGET = 5,        /* fewer kept groups than routed tokens with floor 1     */
     STC_ERR_CUDA = 6,          /* a CUDA runtime call failed                            */
-    STC_ERR_TIMEOUT = 7        /* reserved: no kernel in this library waits             */
+    STC_ERR_TIMEOUT = 7,       /* reserved: no kernel in this library waits             */
+    STC_ERR_SCRATCH_LIMIT = 8  /* problem needs more than the built-in scratch array    */
 } stc_status;
 
 enum { STC_CLS_DROP = 0, STC_CLS_ROUTED = 1, STC_CLS_FULL = 2 };
@@ -126,6 +127,37 @@ int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const v
                          int32_t token_budget, int32_t max_pages, int32_t* page_ids,
                          int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
                          void* stream);
+
+/* stc_quest_select for callers that cannot provide a workspace.  (The paper has
+ * no counterpart: this is a deployment convenience of the library.)
+ *
+ * Who needs it: code that must select pages at a point where it cannot obtain
+ * device memory -- a serving loop whose memory pool is frozen while it runs, a
+ * plugin that is handed only its input and output buffers by the framework that
+ * owns the GPU, a process whose device memory has all been assigned up front.
+ * This call makes no allocation of any kind, on the host or on the device.
+ *
+ * Same operation, arguments, outputs and errors as stc_quest_select, except that
+ * the scratch space (arrival counters + fp32 page scores) is an array built into
+ * the library image: STC_STATIC_SCRATCH_BYTES of device memory on every GPU that
+ * loads the library, held until the process exits.
+ *   - Shapes whose selection workspace (stc_workspace_bytes with
+ *     STC_OP_QUEST_SELECT) exceeds STC_STATIC_SCRATCH_BYTES are refused with
+ *     STC_ERR_SCRATCH_LIMIT before anything is enqueued; with 16-token pages the
+ *     array covers batch * n_kv_heads * ceil(t_cap/16) up to about two million
+ *     pages (e.g. 16 sequences x 8 KV heads x 131072 tokens).
+ *   - The first call made while a given device is current looks up the array's
+ *     address on that device (a runtime query, not an allocation) and remembers
+ *     it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last
+ *     call left in it.  Each call clears the counters it relies on as its first
+ *     enqueued operation, so calls that are ordered on the device (same stream,
+ *     or otherwise serialised) are independent of each other; two calls that
+ *     overlap on the device race on the array and give undefined page lists. */
+#define STC_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t stc_quest_select_static(const stc_shape* shape, const stc_cache* cache, const void* q,
+                                int32_t token_budget, int32_t max_pages, int32_t* page_ids,
+                                int32_t* n_pages, float* scores_opt, void* stream);
 
 /* Sub-token routing and packing (Section 3.3 "Routing mask"; Section 3.4 and
  * Appendix B.1 for the global budget M = N*K; the VLM per-token rule is the

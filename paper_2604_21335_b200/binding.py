@@ -21,11 +21,12 @@ OP_QUEST_SELECT, OP_ROUTE_PACK, OP_DECODE_ATTN = 1, 2, 3
 MODE_GLOBAL, MODE_PER_TOKEN = 0, 1
 CLS_DROP, CLS_ROUTED, CLS_FULL = 0, 1, 2
 STC_OK = 0
+STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static",
 )
 
 
@@ -69,6 +70,8 @@ def load_library():
         lib.stc_build_page_meta.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_int32, C.c_int32, C.c_void_p]
         lib.stc_quest_select.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.stc_quest_select_static.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32,
+                                                C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_route_pack.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                        C.c_int32, C.c_int32, C.c_int32, C.POINTER(_Cache), C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -187,6 +190,19 @@ def quest_select(shape: Shape, cache: Cache, q: torch.Tensor, token_budget: int,
         _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"),
         _ptr(scores, torch.float32, "scores"), _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()),
         "stc_quest_select")
+
+
+def quest_select_static(shape: Shape, cache: Cache, q: torch.Tensor, token_budget: int, page_ids: torch.Tensor,
+                        n_pages: torch.Tensor, scores: Optional[torch.Tensor] = None) -> None:
+    """stc_quest_select without a workspace argument: for callers that cannot
+    allocate device memory where they select pages.  The scratch space is an array
+    inside the library (STATIC_SCRATCH_BYTES per GPU); larger shapes raise StcError
+    with code 8.  Calls must not overlap on the device."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_quest_select_static(
+        C.byref(cs), C.byref(cc), _ptr(q, torch.bfloat16, "q"), token_budget, page_ids.shape[-1],
+        _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"),
+        _ptr(scores, torch.float32, "scores"), _stream()), "stc_quest_select_static")
 
 
 def route_pack(shape: Shape, v: torch.Tensor, scores: torch.Tensor, tok_class: Optional[torch.Tensor],

@@ -47,6 +47,7 @@ const char* stc_status_string(int32_t status) {
         case STC_ERR_BUDGET: return "group budget below one group per routed token";
         case STC_ERR_CUDA: return "CUDA runtime error";
         case STC_ERR_TIMEOUT: return "timeout";
+        case STC_ERR_SCRATCH_LIMIT: return "shape needs more than the built-in scratch array";
         default: return "unknown status";
     }
 }
