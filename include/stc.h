@@ -58,7 +58,7 @@ typedef enum {
     STC_ERR_CAPACITY = 4,      /* packed store too small (device status)                */
     STC_ERR_BUDGET = 5,        /* fewer kept groups than routed tokens with floor 1     */
     STC_ERR_CUDA = 6,          /* a CUDA runtime call failed                            */
-    STC_ERR_TIMEOUT = 7,       /* reserved: no kernel in this library waits             */
+    STC_ERR_TIMEOUT = 7,       /* a bounded device-side wait expired (device status)    */
     STC_ERR_SCRATCH_LIMIT = 8  /* problem needs more than the built-in scratch array    */
 } stc_status;
 
@@ -197,7 +197,13 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
  * bf16 inputs, fp32 accumulation, fp32 outputs; the softmax weights enter the
  * value contraction as a bf16 pair (high + residual part) when the tensor-core
  * path is used (more than one query head per KV head).  lse_opt may be NULL.
- * ws: STC_OP_DECODE_ATTN with arg = max_pages (for page_ids NULL: ceil(T/16)). */
+ * k and v_packed must be 16-byte aligned (pages and packed spans are moved by
+ * bulk asynchronous copies).
+ * ws: STC_OP_DECODE_ATTN with arg = max_pages (for page_ids NULL: ceil(T/16)).
+ * The first int32 of ws is a device status word the call writes: STC_OK, or
+ * STC_ERR_TIMEOUT if a bounded wait for a copy expired on the device (it never
+ * should; out / lse are then unspecified).  It can be read after the stream
+ * has been synchronised. */
 int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const void* q,
                         const int32_t* page_ids, const int32_t* n_pages, int32_t max_pages,
                         float sm_scale, float* out, float* lse_opt, void* ws, size_t ws_bytes,

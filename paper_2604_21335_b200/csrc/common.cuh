@@ -79,7 +79,7 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
                               uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups,
                               int32_t* status, void* ws, cudaStream_t st);
 
-struct AttnPlan { int pages_per_cta, n_splits; };
+struct AttnPlan { int n_workers, slots_cap; };   // warps that share the pages; partial slots per problem
 AttnPlan attn_plan(const Geom& g, int max_pages);
 size_t attn_ws_bytes(const Geom& g, int max_pages);
 cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packed,

@@ -1,30 +1,43 @@
 // Routed decode attention: split-K flash-decode over the selected pages, full
-// width keys, values read from the packed group store and expanded in
-// registers.
+// width keys, values read from the packed group store.
 //
-// Work split: one CTA (4 warps) per (problem, split); a warp owns one 16-token
-// page at a time.  Lane (r = lane/4, c = lane%4) loads, for tokens r and r+8 of
-// the page, the 16-byte chunks c, c+4, c+8, c+12 of the key row (four lanes
-// cover 64 contiguous bytes) and the matching chunks of the value row.  A value
-// chunk whose group was dropped is not loaded at all: the lane substitutes
-// zeros, which is how a dropped group "contributes zero" while its token still
-// counts in the softmax normaliser.  The address of a kept chunk comes from the
-// page's first offset, a 16-lane prefix sum of the tokens' group counts and a
-// popcount of the lower mask bits.
+// Work split.  The (problem, listed page) pairs of the whole call form one flat
+// sequence; it is cut into equal contiguous ranges, one per WARP of a grid that
+// fits the machine in a single wave.  A warp is a complete worker: it streams its
+// pages, keeps its own online-softmax state and, where its range ends inside a
+// problem, writes a partial (max, sum, accumulator) for that problem.  Warps never
+// wait on each other: a per-problem counter of covered pages tells the warp that
+// completes a problem to merge the partials, in slot order, so results are
+// bitwise repeatable.
 //
-// One query head per KV head: dot products and the value update run on the
-// fp32 pipes (2 x 64 FMAs per lane and page).
-// Several query heads per KV head: Q.K^T over the grouped heads is a dense
-// contraction and runs on tensor cores (mma.sync m16n8k16, heads padded to the
-// 16-row operand, key chunks used directly as the col-major operand with the
-// head_dim positions permuted identically on both operands); P.V uses the same
-// instruction with the value chunks transposed in registers (movmatrix); the
-// softmax weights enter as a bf16 high part plus a bf16 residual so the product
-// keeps ~16 bits of the fp32 weight.
+// Data movement.  Each warp owns a ring of kStages shared-memory stages.  A stage
+// holds one page: its 16 key rows (4 KiB, contiguous in HBM) and the packed value
+// groups of its 16 tokens (one contiguous span of the packed store, 0..4 KiB).
+// Lane 0 brings both in with two bulk asynchronous copies (cp.async.bulk, the 1-D
+// TMA path) that signal the stage's mbarrier; the copies for the next kStages-1
+// pages are in flight while the warp computes on the current one, which is what
+// hides HBM latency at 8 warps per SM.  The list entry, sequence length and value
+// offsets a copy needs are fetched 32 pages at a time, one page per lane.
 //
-// Each CTA reduces its warps' (max, sum, acc) states in shared memory and, when
-// the problem is split, writes a partial; the CTA that arrives last at the
-// problem's ticket merges the partials (nobody waits on anybody).
+// A dropped value group is never copied for its own sake and never read: the
+// position of a kept group inside the span follows from the token masks (prefix
+// sum of their popcounts), and a dropped group's operand is a row of zeros, which
+// is how it "contributes zero" while its token still counts in the normaliser.
+//
+// Arithmetic.  One query head per KV head: fp32 FMAs (lane = two tokens x 32
+// dims).  Several query heads per KV head: the two contractions are dense tiles
+// and run on tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate):
+//   S^T[token][head] = K . Q^T      A = key chunks straight from the stage, B = Q
+//   O^T[dim][head]   = V^T . P^T    A = value chunks via ldmatrix.trans with one
+//                                   row address per token (zero row if dropped),
+//                                   B = softmax weights as a bf16 high part plus a
+//                                   bf16 residual (two mma), transposed by movmatrix
+// Both operands of the first product use the same permutation of head_dim
+// positions, so a lane's 16-byte chunk feeds two k-steps without any shuffle.
+//
+// Every wait on an mbarrier is bounded (about a second); a wait that expires
+// records STC_ERR_TIMEOUT in the workspace status word and the warp stops issuing
+// copies, skips its arithmetic and leaves without touching the outputs.
 #include "common.cuh"
 
 namespace stc {
@@ -32,33 +45,84 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
+constexpr int kStages = 3;
 constexpr int kMaxGq = 8;
-constexpr int kTargetCtas = 148 * 4;
-static_assert(kThreads == kHeadDim, "the CTA reductions map one thread to one channel");
+constexpr int kCtasPerSm = 2;
+constexpr int kMinPagesPerWarp = 4;
+constexpr int kMaxSlots = 16;                    // partials per problem the merging warp handles (lane = slot, <= 32)
+constexpr uint32_t kKeyBytes = kPage * kRowBytes;          // 4096
+constexpr uint32_t kStageBytes = 2 * kKeyBytes;            // keys + worst-case value span
+constexpr uint32_t kRingBytes = kWarps * kStages * kStageBytes;
+constexpr uint32_t kSmemBytes = kRingBytes + 64 /* zero row, padded */ + kWarps * kStages * 8 /* mbarriers */;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
-__device__ __forceinline__ void mma_bf16(float& d0, float& d1, float& d2, float& d3, uint32_t a0,
-                                         uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+// ---- PTX wrappers -----------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
-        : "+f"(d0), "+f"(d1), "+f"(d2), "+f"(d3)
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
     return d;
 }
-
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                                  uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for a stage's copies.  False = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+#pragma unroll 1
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+// 1-D bulk copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned; bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
 struct AttnArgs {
-    const uint4* k;
-    const uint4* v_packed;
+    const unsigned char* k;
+    const unsigned char* v_packed;
     const uint16_t* v_mask;
     const uint32_t* v_offs;
     const uint4* q;
@@ -67,343 +131,493 @@ struct AttnArgs {
     const int32_t* seq_len;
     float* out;
     float* lse;
-    float* part_acc;     // [problems][n_splits][Gq][128]
-    float* part_ml;      // [problems][n_splits][Gq][2]
-    unsigned* counters;  // [problems]
+    float* part_acc;     // [problems][slots_cap][Gq][128]
+    float* part_ml;      // [problems][slots_cap][Gq][2]
+    unsigned* counters;  // [problems] pages covered so far
+    int32_t* status;     // one word: STC_OK or STC_ERR_TIMEOUT
     int64_t cap_groups;
-    int Hq, Hkv, Gq, T, max_pages, pages_per_cta, n_splits;
+    long long total;     // problems * max_pages
+    int n_warps;         // workers
+    int slots_cap;
+    int Hq, Hkv, Gq, T, max_pages;
     float scale_log2;    // sm_scale * log2(e)
 };
 
-// Per-page token bookkeeping held by lanes 0..15 (one token each).
-struct TokInfo { uint32_t mask; uint32_t base; };
+// What a lane remembers about one page of the 32-page lookahead window.
+struct PageRef {
+    int page;            // page id, -1 = nothing to attend (past the list, id out of range)
+    int n_valid;         // valid tokens of the page, 1..16
+    uint32_t first;      // first packed group of the page (clipped to the store)
+    uint32_t groups;     // packed groups of the page actually stored
+};
 
 template <int S, bool MMA>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_attn_kernel(const AttnArgs a) {
-    constexpr int OPG = kOctets / S;            // 16-byte chunks per value group
-    constexpr int NH = MMA ? kMaxGq : 1;        // head rows reduced per CTA
-    __shared__ float s_acc[kWarps][NH][kHeadDim];
-    __shared__ float s_m[kWarps][NH], s_l[kWarps][NH];
-    __shared__ int s_last;
+    constexpr int OPG = kOctets / S;             // 16-byte chunks per value group
+    constexpr uint32_t kGroupBytes = OPG * 16;
+    extern __shared__ __align__(128) unsigned char smem[];
 
-    const int problem = blockIdx.x / a.n_splits, split = blockIdx.x - problem * a.n_splits;
-    const int b = problem / a.Hkv, hk = problem - b * a.Hkv;
-    const int len = clamp_len(a.seq_len, b, a.T);
-    const int np = (len + kPage - 1) / kPage;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int r = lane >> 2, c = lane & 3;
-    const int32_t* ids = a.page_ids ? a.page_ids + (size_t)problem * a.max_pages : nullptr;
-    int n_list = ids ? min(max(a.n_pages[problem], 0), a.max_pages) : np;
-    const int begin = split * a.pages_per_cta;
-    const int end = min(n_list, begin + a.pages_per_cta);
-    const int my_count = (end > begin + warp) ? (end - begin - warp + kWarps - 1) / kWarps : 0;
+    const uint32_t ring = smem_u32(smem) + (uint32_t)warp * kStages * kStageBytes;
+    const uint32_t zero_row = smem_u32(smem) + kRingBytes;
+    const uint32_t bars = smem_u32(smem) + kRingBytes + 64 + (uint32_t)warp * kStages * 8;
 
-    const uint4* krows = a.k + (size_t)problem * a.T * kOctets;
-    const uint4* vstore = a.v_packed + (size_t)problem * a.cap_groups * OPG;
-    const int64_t cap_chunks = a.cap_groups * OPG;
-    const uint16_t* masks = a.v_mask + (size_t)problem * a.T;
-    const uint32_t* offs = a.v_offs + (size_t)problem * (a.T + 1);
+    if (tid < 4) reinterpret_cast<uint32_t*>(smem + kRingBytes)[tid] = 0u;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) mbar_init(bars + 8 * s, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();                             // the only CTA-wide barrier: after it warps are independent
 
-    // ---- query operand ------------------------------------------------------
-    // MMA: lane holds chunk c+4j of head row r (zeros past Gq) as A fragments.
-    // MHA: lane holds the same chunks of the single head as floats.
+    const long long w = (long long)blockIdx.x * kWarps + warp;
+    if (w >= a.n_warps) return;
+    const long long x_lo = a.total * w / a.n_warps, x_hi = a.total * (w + 1) / a.n_warps;
+    const int count = (int)(x_hi - x_lo);        // >= 1 by construction (n_warps <= total)
+    const int mp = a.max_pages;
+
+    // ---- lookahead window: lane i describes flat position win_base + i ----------------------
+    PageRef win{-1, 0, 0u, 0u};
+    auto fill_window = [&](long long base) {
+        const long long x = base + lane;
+        win = PageRef{-1, 0, 0u, 0u};
+        if (x < x_hi) {
+            const int p = (int)(x / mp), slot = (int)(x - (long long)p * mp);
+            const int len = clamp_len(a.seq_len, p / a.Hkv, a.T);
+            const int np = (len + kPage - 1) / kPage;
+            int n_list = np, id = slot;
+            if (a.page_ids) {
+                n_list = min(max(a.n_pages[p], 0), mp);
+                id = a.page_ids[(size_t)p * mp + slot];
+            }
+            if (slot < n_list && id >= 0 && id < np) {
+                const int t0 = id * kPage, nv = min(kPage, len - t0);
+                const uint32_t* o = a.v_offs + (size_t)p * (a.T + 1) + t0;
+                const long long ob = min((long long)o[0], (long long)a.cap_groups);
+                const long long oe = min((long long)o[nv], (long long)a.cap_groups);
+                const long long ng = min(oe > ob ? oe - ob : 0LL, (long long)(kPage * S));   // never past the stage
+                win = PageRef{id, nv, (uint32_t)ob, (uint32_t)ng};
+            }
+        }
+    };
+
+    // ---- the pages in flight: a register FIFO, oldest first (uniform across the warp except mask) ----
+    struct InFlight {
+        int nv;              // valid tokens; 0 = nothing to attend at this position
+        uint32_t chunks;     // 16-byte chunks of the value span present in the stage
+        uint32_t mask;       // lanes 0..15: group mask of token `lane`
+    };
+    uint32_t phase = 0;                          // bit s = parity to wait for on stage s
+
+    long long win_base = x_lo;
+    fill_window(win_base);
+    long long x_issue = x_lo;                    // next flat position to bring in
+    int p_issue = (int)(x_lo / mp);              // its problem
+    int slot_issue = (int)(x_lo - (long long)p_issue * mp);
+
+    auto issue = [&](int s) -> InFlight {        // bring position x_issue into stage s
+        InFlight f{0, 0u, 0u};
+        if (x_issue >= x_hi) return f;
+        if (x_issue - win_base >= 32) { win_base = x_issue; fill_window(win_base); }
+        const int src = (int)(x_issue - win_base);
+        const int page = __shfl_sync(0xFFFFFFFFu, win.page, src);
+        const int nv = __shfl_sync(0xFFFFFFFFu, win.n_valid, src);
+        const uint32_t first = __shfl_sync(0xFFFFFFFFu, win.first, src);
+        const uint32_t groups = __shfl_sync(0xFFFFFFFFu, win.groups, src);
+        if (page >= 0) {
+            const size_t row0 = (size_t)p_issue * a.T + (size_t)page * kPage;
+            if (lane < nv) f.mask = a.v_mask[row0 + lane];
+            f.nv = nv;
+            f.chunks = groups * OPG;
+            if (lane == 0) {
+                const uint32_t kb = (uint32_t)nv * kRowBytes, vb = groups * kGroupBytes;
+                const uint32_t bar = bars + 8 * s, dst = ring + (uint32_t)s * kStageBytes;
+                fence_proxy_async();             // the stage's earlier reads precede the new writes
+                mbar_expect_tx(bar, kb + vb);
+                bulk_g2s(dst, a.k + row0 * kRowBytes, kb, bar);
+                if (vb)
+                    bulk_g2s(dst + kKeyBytes,
+                             a.v_packed + ((size_t)p_issue * a.cap_groups + first) * kGroupBytes, vb, bar);
+            }
+        }
+        ++x_issue;
+        if (++slot_issue == mp) { slot_issue = 0; ++p_issue; }
+        return f;
+    };
+
+    // ---- query operand ----------------------------------------------------------------------
+    // MMA: lane (r, c) holds chunks c, c+4, c+8, c+12 of head r (zeros past Gq) = B fragments.
+    // FMA: the same chunks of the single head.
     uint4 qa[4];
-    {
+    auto load_q = [&](int problem) {
+        const int b = problem / a.Hkv, hk = problem - b * a.Hkv;
         const int head = MMA ? r : 0;
         const bool ok = head < a.Gq;
         const uint4* qrow = a.q + ((size_t)b * a.Hq + (size_t)hk * a.Gq + (ok ? head : 0)) * kOctets;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) qa[j] = ok ? qrow[c + 4 * j] : make_uint4(0, 0, 0, 0);
-    }
+        for (int j = 0; j < 4; ++j) qa[j] = ok ? __ldg(qrow + c + 4 * j) : make_uint4(0, 0, 0, 0);
+    };
 
-    float acc[4][4][2];                          // [j][pair][e]: dims 8(c+4j) + 2*pair + e
+    // ---- running state of the current problem -------------------------------------------------
+    // MMA: acc[dt][0..3] = (dim 16dt+r, head 2c), (16dt+r, 2c+1), (16dt+r+8, 2c), (16dt+r+8, 2c+1);
+    //      m_run/l_run[e] belong to head 2c+e (l_run summed over the lane's own tokens only).
+    // FMA: acc[j][2q2+e] -> dim 8(c+4j)+2q2+e, summed over the lane's own two tokens; m_run[0], l_run[0].
+    float acc[8][4];
+    float m_run[2], l_run[2];
+    auto reset_state = [&]() {
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+        for (int i = 0; i < 8; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+        m_run[0] = m_run[1] = -INFINITY;
+        l_run[0] = l_run[1] = 0.f;
+    };
+
+    // ---- one page -----------------------------------------------------------------------------
+    auto compute = [&](int s, const InFlight& f) {
+        const uint32_t kst = ring + (uint32_t)s * kStageBytes, vst = kst + kKeyBytes;
+        const int nv = f.nv;
+        // exclusive prefix (in groups) of the page's token masks, lanes 0..15
+        const uint32_t cnt = __popc(f.mask);
+        uint32_t pre = cnt;
 #pragma unroll
-        for (int p = 0; p < 4; ++p) acc[j][p][0] = acc[j][p][1] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
-    float dz0 = 0.f, dz1 = 0.f;                  // rows 8..15 of the padded head operand
-
-    // Page ids of this warp, 32 at a time: lane i holds the id of the warp's
-    // (n0+i)-th page, so the per-page lookup is a shuffle, not a dependent load.
-    int pid_reg = -1;
-    auto refill = [&](int n0) {
-        const int n = n0 + lane;
-        int p = -1;
-        if (n < my_count) {
-            const int i = begin + warp + n * kWarps;
-            p = ids ? ids[i] : i;
-            if (p < 0 || p >= np) p = -1;
+        for (int d = 1; d < 16; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, pre, d);
+            if (lane >= d) pre += o;
         }
-        pid_reg = p;
-    };
-    auto page_of = [&](int n) -> int {           // n-th page of this warp, -1 if none / invalid
-        if ((n & 31) == 0) refill(n);
-        return __shfl_sync(0xFFFFFFFFu, pid_reg, n & 31);
-    };
-    auto tok_info = [&](int page) -> TokInfo {
-        TokInfo ti{0u, 0u};
-        if (page >= 0) {
-            const int t = page * kPage + lane;
-            if (lane < kPage && t < len) ti.mask = masks[t];
-            ti.base = offs[page * kPage];
-        }
-        return ti;
-    };
+        pre -= cnt;
 
-    int page = page_of(0);
-    TokInfo ti = tok_info(page);
-#pragma unroll 1
-    for (int n = 0; n < my_count; ++n) {
-        const int page_next = page_of(n + 1);
-        const TokInfo ti_next = tok_info(page_next);
-        if (page >= 0) {
-            const int t0 = page * kPage;
-            // ---- key loads ----------------------------------------------------
+        if constexpr (MMA) {
+            // S^T = K . Q^T : rows = tokens (r, r+8), columns = heads (2c, 2c+1)
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 k0 = lds16(kst + (uint32_t)r * kRowBytes + (uint32_t)(c + 4 * j) * 16u);
+                const uint4 k1 = lds16(kst + (uint32_t)(r + 8) * kRowBytes + (uint32_t)(c + 4 * j) * 16u);
+                mma_bf16(s0, k0.x, k1.x, k0.y, k1.y, qa[j].x, qa[j].y);
+                mma_bf16(s1, k0.z, k1.z, k0.w, k1.w, qa[j].z, qa[j].w);
+            }
+            const bool v0 = r < nv, v1 = r + 8 < nv;
+            float sv[4];
+            sv[0] = v0 ? (s0[0] + s1[0]) * a.scale_log2 : -INFINITY;
+            sv[1] = v0 ? (s0[1] + s1[1]) * a.scale_log2 : -INFINITY;
+            sv[2] = v1 ? (s0[2] + s1[2]) * a.scale_log2 : -INFINITY;
+            sv[3] = v1 ? (s0[3] + s1[3]) * a.scale_log2 : -INFINITY;
+            float pm0 = fmaxf(sv[0], sv[2]), pm1 = fmaxf(sv[1], sv[3]);
+#pragma unroll
+            for (int d = 4; d < 32; d <<= 1) {
+                pm0 = fmaxf(pm0, __shfl_xor_sync(0xFFFFFFFFu, pm0, d));
+                pm1 = fmaxf(pm1, __shfl_xor_sync(0xFFFFFFFFu, pm1, d));
+            }
+            const float mn0 = fmaxf(m_run[0], pm0), mn1 = fmaxf(m_run[1], pm1);   // finite: token 0 is valid
+            const float al0 = exp2f(m_run[0] - mn0), al1 = exp2f(m_run[1] - mn1);
+            const float p0 = exp2f(sv[0] - mn0), p1 = exp2f(sv[1] - mn1);
+            const float p2 = exp2f(sv[2] - mn0), p3 = exp2f(sv[3] - mn1);
+            l_run[0] = fmaf(l_run[0], al0, p0 + p2);
+            l_run[1] = fmaf(l_run[1], al1, p1 + p3);
+            m_run[0] = mn0; m_run[1] = mn1;
+            // P^T as B fragments: high bf16 part and bf16 residual
+            const uint32_t wh0 = pack_bf16(p0, p1), wh1 = pack_bf16(p2, p3);
+            const uint32_t wl0 = pack_bf16(p0 - bf16lo(wh0), p1 - bf16hi(wh0));
+            const uint32_t wl1 = pack_bf16(p2 - bf16lo(wh1), p3 - bf16hi(wh1));
+            const uint32_t bh0 = movmatrix_trans(wh0), bh1 = movmatrix_trans(wh1);
+            const uint32_t bl0 = movmatrix_trans(wl0), bl1 = movmatrix_trans(wl1);
+            // value rows: this lane addresses token tau, chunk 2dt + hb of every dim tile
+            const int tau = (lane & 7) + 8 * (lane >> 4), hb = (lane >> 3) & 1;
+            const uint32_t m = __shfl_sync(0xFFFFFFFFu, f.mask, tau);
+            const uint32_t base = __shfl_sync(0xFFFFFFFFu, pre, tau) * OPG;
+            const uint32_t limit = f.chunks;
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+                const int oct = 2 * dt + hb, grp = oct / OPG;
+                const uint32_t idx = base + __popc(m & ((1u << grp) - 1u)) * OPG + (uint32_t)(oct % OPG);
+                const bool kept = ((m >> grp) & 1u) && idx < limit;
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4_trans(kept ? vst + idx * 16u : zero_row, a0, a1, a2, a3);
+                acc[dt][0] *= al0; acc[dt][1] *= al1; acc[dt][2] *= al0; acc[dt][3] *= al1;
+                mma_bf16(acc[dt], a0, a1, a2, a3, bh0, bh1);
+                mma_bf16(acc[dt], a0, a1, a2, a3, bl0, bl1);
+            }
+        } else {
+            // one head on the fp32 pipes: lane = tokens r, r+8 x chunks c, c+4, c+8, c+12
+            float sd[2];
             uint4 kr[2][4];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int t = t0 + r + 8 * hf;
-                const uint4* row = krows + (size_t)t * kOctets;
+            for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    kr[hf][j] = (t < len) ? ldg_nc16(row + c + 4 * j) : make_uint4(0, 0, 0, 0);
-            }
-            // ---- value loads, dropped groups become zeros ------------------------
-            uint32_t cnt = __popc(ti.mask), pre = cnt;
+                    kr[hf][j] = lds16(kst + (uint32_t)(r + 8 * hf) * kRowBytes + (uint32_t)(c + 4 * j) * 16u);
 #pragma unroll
-            for (int d = 1; d < 16; d <<= 1) {
-                uint32_t o = __shfl_up_sync(0xFFFFFFFFu, pre, d);
-                if (lane >= d) pre += o;
+            for (int hf = 0; hf < 2; ++hf) {
+                float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    d0 = fmaf(bf16lo(qa[j].x), bf16lo(kr[hf][j].x), d0);
+                    d1 = fmaf(bf16hi(qa[j].x), bf16hi(kr[hf][j].x), d1);
+                    d0 = fmaf(bf16lo(qa[j].y), bf16lo(kr[hf][j].y), d0);
+                    d1 = fmaf(bf16hi(qa[j].y), bf16hi(kr[hf][j].y), d1);
+                    d0 = fmaf(bf16lo(qa[j].z), bf16lo(kr[hf][j].z), d0);
+                    d1 = fmaf(bf16hi(qa[j].z), bf16hi(kr[hf][j].z), d1);
+                    d0 = fmaf(bf16lo(qa[j].w), bf16lo(kr[hf][j].w), d0);
+                    d1 = fmaf(bf16hi(qa[j].w), bf16hi(kr[hf][j].w), d1);
+                }
+                float d = d0 + d1;
+                d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
+                d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
+                sd[hf] = (r + 8 * hf < nv) ? d * a.scale_log2 : -INFINITY;
             }
-            pre -= cnt;                           // exclusive, lanes 0..15
+            float pm = fmaxf(sd[0], sd[1]);
+#pragma unroll
+            for (int d = 4; d < 32; d <<= 1) pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, d));
+            const float mn = fmaxf(m_run[0], pm);
+            const float al = exp2f(m_run[0] - mn);
+            const float p0 = exp2f(sd[0] - mn), p1 = exp2f(sd[1] - mn);
+            l_run[0] = fmaf(l_run[0], al, p0 + p1);
+            m_run[0] = mn;
+            const uint32_t limit = f.chunks;
             uint4 vr[2][4];
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-                const uint32_t m = __shfl_sync(0xFFFFFFFFu, ti.mask, r + 8 * hf);
-                const uint32_t first = ti.base + __shfl_sync(0xFFFFFFFFu, pre, r + 8 * hf);
+                const uint32_t m = __shfl_sync(0xFFFFFFFFu, f.mask, r + 8 * hf);
+                const uint32_t base = __shfl_sync(0xFFFFFFFFu, pre, r + 8 * hf) * OPG;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int oct = c + 4 * j, grp = oct / OPG;
-                    const int64_t chunk = (int64_t)(first + __popc(m & ((1u << grp) - 1u))) * OPG + (oct % OPG);
-                    vr[hf][j] = (((m >> grp) & 1u) && chunk < cap_chunks) ? ldg_nc16(vstore + chunk)
-                                                                          : make_uint4(0, 0, 0, 0);
+                    const uint32_t idx = base + __popc(m & ((1u << grp) - 1u)) * OPG + (uint32_t)(oct % OPG);
+                    const bool kept = ((m >> grp) & 1u) && idx < limit;
+                    vr[hf][j] = kept ? lds16(vst + idx * 16u) : make_uint4(0, 0, 0, 0);
                 }
             }
-
-            if constexpr (MMA) {
-                // ---- S = Q.K^T on tensor cores: rows = heads, cols = tokens -------
-                float s[2][4];
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    s[hf][0] = s[hf][1] = s[hf][2] = s[hf][3] = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        mma_bf16(s[hf][0], s[hf][1], s[hf][2], s[hf][3], qa[j].x, 0u, qa[j].y, 0u,
-                                 kr[hf][j].x, kr[hf][j].y);
-                        mma_bf16(s[hf][0], s[hf][1], s[hf][2], s[hf][3], qa[j].z, 0u, qa[j].w, 0u,
-                                 kr[hf][j].z, kr[hf][j].w);
-                    }
-                }
-                // lane: head r, tokens 8hf + 2c + e
-                float sv[2][2], pmax = -INFINITY;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const bool valid = t0 + 8 * hf + 2 * c + e < len;
-                        sv[hf][e] = valid ? s[hf][e] * a.scale_log2 : -INFINITY;
-                        pmax = fmaxf(pmax, sv[hf][e]);
-                    }
-                pmax = fmaxf(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, 1));
-                pmax = fmaxf(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, 2));
-                const float m_new = fmaxf(m_run, pmax);
-                const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                const float alpha = exp2f(m_run - m_use);
-                float p[2][2];
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) p[hf][e] = exp2f(sv[hf][e] - m_use);
-                l_run = l_run * alpha + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
-                m_run = m_new;
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-#pragma unroll
-                    for (int q2 = 0; q2 < 4; ++q2) { acc[j][q2][0] *= alpha; acc[j][q2][1] *= alpha; }
-                // weights as bf16 high part + residual (A fragments: k = token)
-                const uint32_t ph0 = pack_bf16(p[0][0], p[0][1]), ph2 = pack_bf16(p[1][0], p[1][1]);
-                const uint32_t pl0 = pack_bf16(p[0][0] - bf16lo(ph0), p[0][1] - bf16hi(ph0));
-                const uint32_t pl2 = pack_bf16(p[1][0] - bf16lo(ph2), p[1][1] - bf16hi(ph2));
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t v0[4] = {vr[0][j].x, vr[0][j].y, vr[0][j].z, vr[0][j].w};
-                    const uint32_t v1[4] = {vr[1][j].x, vr[1][j].y, vr[1][j].z, vr[1][j].w};
-#pragma unroll
-                    for (int q2 = 0; q2 < 4; ++q2) {
-                        const uint32_t b0 = movmatrix_trans(v0[q2]);   // tokens 0..7  x 8 dims
-                        const uint32_t b1 = movmatrix_trans(v1[q2]);   // tokens 8..15 x 8 dims
-                        mma_bf16(acc[j][q2][0], acc[j][q2][1], dz0, dz1, ph0, 0u, ph2, 0u, b0, b1);
-                        mma_bf16(acc[j][q2][0], acc[j][q2][1], dz0, dz1, pl0, 0u, pl2, 0u, b0, b1);
-                    }
-                }
-            } else {
-                // ---- one head: fp32 pipes ----------------------------------------
-                float sdot[2];
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    float d = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        d = fmaf(bf16lo(qa[j].x), bf16lo(kr[hf][j].x), d);
-                        d = fmaf(bf16hi(qa[j].x), bf16hi(kr[hf][j].x), d);
-                        d = fmaf(bf16lo(qa[j].y), bf16lo(kr[hf][j].y), d);
-                        d = fmaf(bf16hi(qa[j].y), bf16hi(kr[hf][j].y), d);
-                        d = fmaf(bf16lo(qa[j].z), bf16lo(kr[hf][j].z), d);
-                        d = fmaf(bf16hi(qa[j].z), bf16hi(kr[hf][j].z), d);
-                        d = fmaf(bf16lo(qa[j].w), bf16lo(kr[hf][j].w), d);
-                        d = fmaf(bf16hi(qa[j].w), bf16hi(kr[hf][j].w), d);
-                    }
-                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-                    d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
-                    sdot[hf] = (t0 + r + 8 * hf < len) ? d * a.scale_log2 : -INFINITY;
-                }
-                float pmax = fmaxf(sdot[0], sdot[1]);
-                pmax = fmaxf(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, 4));
-                pmax = fmaxf(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, 8));
-                pmax = fmaxf(pmax, __shfl_xor_sync(0xFFFFFFFFu, pmax, 16));
-                const float m_new = fmaxf(m_run, pmax);
-                const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-                const float alpha = exp2f(m_run - m_use);
-                const float p0 = exp2f(sdot[0] - m_use), p1 = exp2f(sdot[1] - m_use);
-                l_run = l_run * alpha + p0 + p1;   // per token-lane; summed over r at the end
-                m_run = m_new;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t v0[4] = {vr[0][j].x, vr[0][j].y, vr[0][j].z, vr[0][j].w};
-                    const uint32_t v1[4] = {vr[1][j].x, vr[1][j].y, vr[1][j].z, vr[1][j].w};
-#pragma unroll
-                    for (int q2 = 0; q2 < 4; ++q2) {
-                        acc[j][q2][0] = fmaf(p1, bf16lo(v1[q2]), fmaf(p0, bf16lo(v0[q2]), acc[j][q2][0] * alpha));
-                        acc[j][q2][1] = fmaf(p1, bf16hi(v1[q2]), fmaf(p0, bf16hi(v0[q2]), acc[j][q2][1] * alpha));
-                    }
-                }
-            }
-        }
-        page = page_next;
-        ti = ti_next;
-    }
-
-    // ---- warp state -> shared memory -----------------------------------------
-    if constexpr (MMA) {
-        l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 1);
-        l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, 2);
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int q2 = 0; q2 < 4; ++q2)
-                *reinterpret_cast<float2*>(&s_acc[warp][r][8 * (c + 4 * j) + 2 * q2]) =
-                    make_float2(acc[j][q2][0], acc[j][q2][1]);
-        if (c == 0) { s_m[warp][r] = m_run; s_l[warp][r] = l_run; }
-    } else {
-#pragma unroll
-        for (int d = 4; d < 32; d <<= 1) {
-            l_run += __shfl_xor_sync(0xFFFFFFFFu, l_run, d);
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t u0[4] = {vr[0][j].x, vr[0][j].y, vr[0][j].z, vr[0][j].w};
+                const uint32_t u1[4] = {vr[1][j].x, vr[1][j].y, vr[1][j].z, vr[1][j].w};
 #pragma unroll
                 for (int q2 = 0; q2 < 4; ++q2) {
-                    acc[j][q2][0] += __shfl_xor_sync(0xFFFFFFFFu, acc[j][q2][0], d);
-                    acc[j][q2][1] += __shfl_xor_sync(0xFFFFFFFFu, acc[j][q2][1], d);
+                    float& lo = acc[2 * j + (q2 >> 1)][2 * (q2 & 1)];
+                    float& hi = acc[2 * j + (q2 >> 1)][2 * (q2 & 1) + 1];
+                    lo = fmaf(p1, bf16lo(u1[q2]), fmaf(p0, bf16lo(u0[q2]), lo * al));
+                    hi = fmaf(p1, bf16hi(u1[q2]), fmaf(p0, bf16hi(u0[q2]), hi * al));
                 }
+            }
         }
-        if (r == 0) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int q2 = 0; q2 < 4; ++q2)
-                    *reinterpret_cast<float2*>(&s_acc[warp][0][8 * (c + 4 * j) + 2 * q2]) =
-                        make_float2(acc[j][q2][0], acc[j][q2][1]);
-            if (c == 0) { s_m[warp][0] = m_run; s_l[warp][0] = l_run; }
-        }
-    }
-    __syncthreads();
+    };
 
-    // ---- CTA reduction: thread = one channel, loop over heads -----------------
-    const int gq = MMA ? a.Gq : 1;
+    // ---- end of a problem segment: output, or partial + ticket + merge ---------------------
     const float ln2 = 0.6931471805599453f;
-    for (int h = 0; h < gq; ++h) {
-        float M = -INFINITY;
+    auto finish = [&](int problem, int covered) {
+        const int b = problem / a.Hkv, hk = problem - b * a.Hkv;
+        const size_t row_base = (size_t)b * a.Hq + (size_t)hk * a.Gq;
+        // totals of the normaliser over the lanes that share a head column / the single head
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, s_m[w][h]);
-        float L = 0.f, o = 0.f;
+        for (int d = 4; d < 32; d <<= 1) {
+            l_run[0] += __shfl_xor_sync(0xFFFFFFFFu, l_run[0], d);
+            if (MMA) l_run[1] += __shfl_xor_sync(0xFFFFFFFFu, l_run[1], d);
+        }
+        if constexpr (!MMA) {
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const float mw = s_m[w][h];
-            const float sc = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
-            L = fmaf(s_l[w][h], sc, L);
-            o = fmaf(s_acc[w][h][tid], sc, o);
+            for (int d = 4; d < 32; d <<= 1)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[i][e] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][e], d);
         }
-        if (a.n_splits == 1) {
-            const size_t row = (size_t)b * a.Hq + (size_t)hk * a.Gq + h;
-            a.out[row * kHeadDim + tid] = L > 0.f ? o / L : 0.f;
-            if (a.lse && tid == 0) a.lse[row] = L > 0.f ? (M + log2f(L)) * ln2 : -INFINITY;
-        } else {
-            const size_t slot = ((size_t)problem * a.n_splits + split) * a.Gq + h;
-            a.part_acc[slot * kHeadDim + tid] = o;
-            if (tid == 0) { a.part_ml[slot * 2] = M; a.part_ml[slot * 2 + 1] = L; }
-        }
-    }
-    if (a.n_splits == 1) return;
+        const bool whole = covered == mp;         // this warp saw the whole problem: no partial needed
+        // first / count of the workers that overlap this problem (closed forms of the equal split)
+        const long long A = (long long)problem * mp;
+        const long long first = ((A + 1) * a.n_warps + a.total - 1) / a.total - 1;
+        const long long last = ((A + mp) * a.n_warps + a.total - 1) / a.total - 1;
+        const int n_slots = (int)(last - first + 1);
+        const size_t slot0 = ((size_t)problem * a.slots_cap) * a.Gq;
+        const size_t slot = slot0 + (size_t)(w - first) * a.Gq;
 
-    // ---- last CTA of the problem merges the partials ---------------------------
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(&a.counters[problem], 1u) == (unsigned)(a.n_splits - 1));
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    for (int h = 0; h < gq; ++h) {
-        const size_t slot0 = (size_t)problem * a.n_splits * a.Gq + h;
-        float M = -INFINITY;
-        for (int s = 0; s < a.n_splits; ++s) M = fmaxf(M, __ldcg(a.part_ml + (slot0 + (size_t)s * a.Gq) * 2));
-        float L = 0.f, o = 0.f;
-        for (int s = 0; s < a.n_splits; ++s) {
-            const size_t slot = slot0 + (size_t)s * a.Gq;
-            const float ms = __ldcg(a.part_ml + slot * 2);
-            const float sc = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
-            L = fmaf(__ldcg(a.part_ml + slot * 2 + 1), sc, L);
-            o = fmaf(__ldcg(a.part_acc + slot * kHeadDim + tid), sc, o);
+        if constexpr (MMA) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int h = 2 * c + e;
+                if (h >= a.Gq) continue;
+                if (whole) {
+                    const float inv = l_run[e] > 0.f ? 1.f / l_run[e] : 0.f;
+                    float* o = a.out + (row_base + h) * kHeadDim;
+#pragma unroll
+                    for (int dt = 0; dt < 8; ++dt) {
+                        o[16 * dt + r] = acc[dt][e] * inv;
+                        o[16 * dt + r + 8] = acc[dt][2 + e] * inv;
+                    }
+                    if (a.lse && r == 0)
+                        a.lse[row_base + h] = l_run[e] > 0.f ? (m_run[e] + log2f(l_run[e])) * ln2 : -INFINITY;
+                } else {
+                    float* o = a.part_acc + (slot + h) * kHeadDim;
+#pragma unroll
+                    for (int dt = 0; dt < 8; ++dt) {
+                        o[16 * dt + r] = acc[dt][e];
+                        o[16 * dt + r + 8] = acc[dt][2 + e];
+                    }
+                    if (r == 0) { a.part_ml[(slot + h) * 2] = m_run[e]; a.part_ml[(slot + h) * 2 + 1] = l_run[e]; }
+                }
+            }
+        } else {
+            if (r == 0) {                          // lanes 0..3 hold the reduced 128 channels
+                const float inv = l_run[0] > 0.f ? 1.f / l_run[0] : 0.f;
+                float* o = whole ? a.out + row_base * kHeadDim : a.part_acc + slot * kHeadDim;
+                const float sc = whole ? inv : 1.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float4 lo = make_float4(acc[2 * j][0] * sc, acc[2 * j][1] * sc, acc[2 * j][2] * sc, acc[2 * j][3] * sc);
+                    float4 hi = make_float4(acc[2 * j + 1][0] * sc, acc[2 * j + 1][1] * sc, acc[2 * j + 1][2] * sc,
+                                            acc[2 * j + 1][3] * sc);
+                    *reinterpret_cast<float4*>(o + 8 * (c + 4 * j)) = lo;
+                    *reinterpret_cast<float4*>(o + 8 * (c + 4 * j) + 4) = hi;
+                }
+                if (c == 0) {
+                    if (whole) {
+                        if (a.lse) a.lse[row_base] = l_run[0] > 0.f ? (m_run[0] + log2f(l_run[0])) * ln2 : -INFINITY;
+                    } else {
+                        a.part_ml[slot * 2] = m_run[0];
+                        a.part_ml[slot * 2 + 1] = l_run[0];
+                    }
+                }
+            }
         }
-        const size_t row = (size_t)b * a.Hq + (size_t)hk * a.Gq + h;
-        a.out[row * kHeadDim + tid] = L > 0.f ? o / L : 0.f;
-        if (a.lse && tid == 0) a.lse[row] = L > 0.f ? (M + log2f(L)) * ln2 : -INFINITY;
+        if (whole) return;
+
+        // ticket: the worker that completes the problem's page count merges, in slot order
+        __threadfence();
+        __syncwarp();
+        unsigned old = 0;
+        if (lane == 0) old = atomicAdd(&a.counters[problem], (unsigned)covered);
+        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        if (old + (unsigned)covered != (unsigned)mp) return;
+        __threadfence();
+        // (1) lane = slot: all (max, sum) pairs of the problem in one round of loads (indices
+        //     clamped, so nothing is conditional), then per head the global max, each slot's
+        //     weight 2^(m - M) and the total of the normaliser
+        const int sl_mine = min(lane, n_slots - 1);
+        float2 ml[kMaxGq];
+#pragma unroll
+        for (int h = 0; h < kMaxGq; ++h)
+            ml[h] = __ldcg(reinterpret_cast<const float2*>(a.part_ml) + slot0 + (size_t)sl_mine * a.Gq + min(h, a.Gq - 1));
+        float wgt[kMaxGq], M[kMaxGq], L[kMaxGq];
+#pragma unroll
+        for (int h = 0; h < kMaxGq; ++h) {
+            const float m = lane < n_slots ? ml[h].x : -INFINITY;
+            float mx = m;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
+            wgt[h] = (m == -INFINITY) ? 0.f : exp2f(m - mx);
+            float ls = lane < n_slots ? ml[h].y * wgt[h] : 0.f;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, d);
+            M[h] = mx; L[h] = ls;
+        }
+        // (2) weighted sums in slot order; each lane owns 4 channels of every head
+        float4 o[kMaxGq];
+#pragma unroll
+        for (int h = 0; h < kMaxGq; ++h) o[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+        for (int sl = 0; sl < n_slots; ++sl) {
+#pragma unroll
+            for (int h = 0; h < kMaxGq; ++h) {
+                const size_t ps = slot0 + (size_t)sl * a.Gq + min(h, a.Gq - 1);
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + ps * kHeadDim) + lane);
+                const float sc = __shfl_sync(0xFFFFFFFFu, wgt[h], sl);
+                o[h].x = fmaf(v.x, sc, o[h].x); o[h].y = fmaf(v.y, sc, o[h].y);
+                o[h].z = fmaf(v.z, sc, o[h].z); o[h].w = fmaf(v.w, sc, o[h].w);
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < kMaxGq; ++h) {
+            if (h >= a.Gq) continue;
+            const float inv = L[h] > 0.f ? 1.f / L[h] : 0.f;
+            reinterpret_cast<float4*>(a.out + (row_base + h) * kHeadDim)[lane] =
+                make_float4(o[h].x * inv, o[h].y * inv, o[h].z * inv, o[h].w * inv);
+            if (a.lse && lane == 0) a.lse[row_base + h] = L[h] > 0.f ? (M[h] + log2f(L[h])) * ln2 : -INFINITY;
+        }
+    };
+
+    // ---- main loop ----------------------------------------------------------------------------
+    InFlight f0 = issue(0), f1 = issue(1), f2 = issue(2);
+    static_assert(kStages == 3, "the in-flight FIFO is written out for three stages");
+
+    int p_cur = (int)(x_lo / mp);
+    int slot_cur = (int)(x_lo - (long long)p_cur * mp);
+    int seg_begin_slot = slot_cur;
+    load_q(p_cur);
+    reset_state();
+    int s = 0;
+#pragma unroll 1
+    for (int n = 0; n < count; ++n) {
+        if (f0.nv > 0) {                          // uniform across the warp
+            const uint32_t par = (phase >> s) & 1u;
+            phase ^= 1u << s;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(bars + 8 * s, par))) {
+                // A copy did not land in time.  Report it, give the copies still in flight
+                // one more bounded wait each so they do not land in a dead CTA's memory,
+                // and leave; the outputs this worker owes stay unwritten.
+                if (lane == 0) atomicExch(a.status, (int)STC_ERR_TIMEOUT);
+                const int s1 = s + 1 == kStages ? 0 : s + 1, s2 = s1 + 1 == kStages ? 0 : s1 + 1;
+                if (f1.nv > 0) mbar_wait(bars + 8 * s1, (phase >> s1) & 1u);
+                if (f2.nv > 0) mbar_wait(bars + 8 * s2, (phase >> s2) & 1u);
+                return;
+            }
+            compute(s, f0);
+        }
+        __syncwarp();
+        f0 = f1; f1 = f2; f2 = issue(s);
+        s = s + 1 == kStages ? 0 : s + 1;
+        if (++slot_cur == mp) {                   // problem boundary inside the range
+            finish(p_cur, mp - seg_begin_slot);
+            ++p_cur; slot_cur = 0; seg_begin_slot = 0;
+            if (n + 1 < count) { load_q(p_cur); reset_state(); }
+        }
     }
+    if (slot_cur != 0) finish(p_cur, slot_cur - seg_begin_slot);
+}
+
+// out = 0, lse = -inf for every head: the call has nothing to attend.
+__global__ void attn_empty_kernel(float* __restrict__ out, float* __restrict__ lse, int rows) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < rows * kHeadDim) out[i] = 0.f;
+    if (lse && i < rows) lse[i] = -INFINITY;
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
 }  // namespace
 
+// Workers (warps) and partial slots per problem.  Sized from max_pages only, so the
+// workspace query and the launch agree; independent of the device so that the
+// workspace size can be asked for without one.
 AttnPlan attn_plan(const Geom& g, int max_pages) {
     AttnPlan p;
-    max_pages = max_pages < 1 ? 1 : max_pages;
-    const int problems = g.problems < 1 ? 1 : g.problems;
-    int splits = (kTargetCtas + problems - 1) / problems;
-    const int max_splits = (max_pages + kWarps - 1) / kWarps;
-    splits = splits < 1 ? 1 : (splits > max_splits ? max_splits : splits);
-    int ppc = (max_pages + splits - 1) / splits;
-    ppc = (ppc + kWarps - 1) / kWarps * kWarps;
-    p.pages_per_cta = ppc;
-    p.n_splits = (max_pages + ppc - 1) / ppc;
+    const long long mp = max_pages < 1 ? 1 : max_pages;
+    const long long total = (long long)(g.problems < 1 ? 1 : g.problems) * mp;
+    long long workers = (total + kMinPagesPerWarp - 1) / kMinPagesPerWarp;
+    const long long wave = 148LL * kCtasPerSm * kWarps;
+    if (workers > wave) workers = wave;
+    const long long by_slots = (long long)(kMaxSlots - 1) * (g.problems < 1 ? 1 : g.problems);
+    if (workers > by_slots) workers = by_slots;  // keeps ceil(workers / problems) + 1 <= kMaxSlots
+    if (workers < 1) workers = 1;
+    p.n_workers = (int)workers;
+    p.slots_cap = (int)((workers + g.problems - 1) / (g.problems < 1 ? 1 : g.problems)) + 1;
     return p;
 }
 
 size_t attn_ws_bytes(const Geom& g, int max_pages) {
     const AttnPlan p = attn_plan(g, max_pages);
-    const size_t slots = (size_t)g.problems * p.n_splits * g.Gq;
-    return align256((size_t)g.problems * 4) + align256(slots * kHeadDim * 4) + align256(slots * 2 * 4);
+    const size_t slots = (size_t)g.problems * p.slots_cap * g.Gq;
+    return 256 + align256((size_t)g.problems * 4) + align256(slots * kHeadDim * 4) + align256(slots * 2 * 4);
 }
 
 cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packed,
@@ -412,17 +626,25 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
                                int max_pages, float sm_scale, float* out, float* lse, void* ws,
                                cudaStream_t st) {
     if (g.problems == 0) return cudaSuccess;
+    const int rows = g.B * g.Hq;
+    char* wsp = static_cast<char*>(ws);
+    if (max_pages < 1 || g.T == 0) {
+        cudaError_t e = cudaMemsetAsync(wsp, 0, 4, st);
+        if (e != cudaSuccess) return e;
+        attn_empty_kernel<<<(rows * kHeadDim + 255) / 256, 256, 0, st>>>(out, lse, rows);
+        return cudaGetLastError();
+    }
     const AttnPlan p = attn_plan(g, max_pages);
-    const size_t slots = (size_t)g.problems * p.n_splits * g.Gq;
+    const size_t slots = (size_t)g.problems * p.slots_cap * g.Gq;
     AttnArgs a;
-    char* w = static_cast<char*>(ws);
-    a.counters = reinterpret_cast<unsigned*>(w);
-    w += align256((size_t)g.problems * 4);
+    a.status = reinterpret_cast<int32_t*>(wsp);
+    a.counters = reinterpret_cast<unsigned*>(wsp + 256);
+    char* w = wsp + 256 + align256((size_t)g.problems * 4);
     a.part_acc = reinterpret_cast<float*>(w);
     w += align256(slots * kHeadDim * 4);
     a.part_ml = reinterpret_cast<float*>(w);
-    a.k = static_cast<const uint4*>(k);
-    a.v_packed = static_cast<const uint4*>(v_packed);
+    a.k = static_cast<const unsigned char*>(k);
+    a.v_packed = static_cast<const unsigned char*>(v_packed);
     a.v_mask = v_mask;
     a.v_offs = v_offs;
     a.q = static_cast<const uint4*>(q);
@@ -432,22 +654,29 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
     a.out = out;
     a.lse = lse;
     a.cap_groups = cap_groups;
+    a.total = (long long)g.problems * max_pages;
+    a.n_warps = p.n_workers;
+    a.slots_cap = p.slots_cap;
     a.Hq = g.Hq; a.Hkv = g.Hkv; a.Gq = g.Gq; a.T = g.T;
     a.max_pages = max_pages;
-    a.pages_per_cta = p.pages_per_cta;
-    a.n_splits = p.n_splits;
     a.scale_log2 = sm_scale * 1.4426950408889634f;
-    if (p.n_splits > 1) {
-        cudaError_t e = cudaMemsetAsync(a.counters, 0, (size_t)g.problems * 4, st);
-        if (e != cudaSuccess) return e;
-    }
-    const long long n_cta = (long long)g.problems * p.n_splits;
-    if (n_cta > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    // status word + page counters start at zero
+    cudaError_t e = cudaMemsetAsync(wsp, 0, 256 + (size_t)g.problems * 4, st);
+    if (e != cudaSuccess) return e;
+    const int n_cta = (p.n_workers + kWarps - 1) / kWarps;
+    (void)sm_count;
     const bool mma = g.Gq > 1;
-#define STC_ATTN(S_)                                                                         \
-    case S_:                                                                                 \
-        if (mma) decode_attn_kernel<S_, true><<<(unsigned)n_cta, kThreads, 0, st>>>(a);      \
-        else     decode_attn_kernel<S_, false><<<(unsigned)n_cta, kThreads, 0, st>>>(a);     \
+#define STC_ATTN(S_)                                                                                    \
+    case S_:                                                                                            \
+        if (mma) {                                                                                      \
+            cudaFuncSetAttribute(decode_attn_kernel<S_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 (int)kSmemBytes);                                                      \
+            decode_attn_kernel<S_, true><<<n_cta, kThreads, kSmemBytes, st>>>(a);                       \
+        } else {                                                                                        \
+            cudaFuncSetAttribute(decode_attn_kernel<S_, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 (int)kSmemBytes);                                                      \
+            decode_attn_kernel<S_, false><<<n_cta, kThreads, kSmemBytes, st>>>(a);                      \
+        }                                                                                               \
         break;
     switch (g.S) {
         STC_ATTN(4) STC_ATTN(8) STC_ATTN(16)

@@ -142,6 +142,8 @@ int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const vo
     if (max_pages > g.P && !page_ids) return STC_ERR_INVALID_ARG;
     if (g.T > 0 && (!cache->k || !cache->v_packed || !cache->v_mask || !cache->v_offs || cache->cap_groups < 0))
         return STC_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v_packed)) & 15u) != 0)
+        return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, attn_ws_bytes(g, max_pages));
     if (rc != STC_OK) return rc;
     return cuda_rc(launch_decode_attn(g, cache->k, cache->v_packed, cache->v_mask, cache->v_offs,

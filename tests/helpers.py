@@ -68,6 +68,7 @@ def gpu_pipeline(w, d, seq_len=None, budget=None, k_nominal=None, min_per_token=
     ws_a.fill_(0xEF)
     P.decode_attn(shape, cache, q, page_ids, n_pages, SM_SCALE, out, ws_a, lse=lse)
     torch.cuda.synchronize()
+    assert int(ws_a[:4].view(torch.int32)[0]) == 0, "device status word of stc_decode_attn"
     res["out"], res["lse"] = out, lse
     return res
 
