@@ -26,11 +26,10 @@
 // partial wave.  Inside a problem each lane keeps a private ring of 16-byte
 // cp.async copies running kDepth units ahead; nothing waits on another thread.
 // When a CTA leaves a problem it adds the units it covered to the problem's
-// counter; whoever completes the count (no waiting) selects the pages: bitwise
-// binary search for the k-th largest order-preserving key held in registers (no
-// atomics, so hot histogram bins cannot serialise it), then an ordered
-// compaction that emits ids ascending and resolves ties at the threshold in
-// favour of lower page ids.
+// counter; whoever completes the count (no waiting) selects the pages: radix
+// select of the k-th largest order-preserving key on the bits the problem's keys
+// actually differ in, then an ordered compaction that emits ids ascending and
+// resolves ties at the threshold in favour of lower page ids (see block_topk).
 #include "common.cuh"
 
 namespace stc {
@@ -41,8 +40,6 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kCtasPerSm = 2;
 constexpr int kDepth = 8;                    // units in flight per lane (32 B each)
 constexpr size_t kRingBytes = (size_t)kDepth * kThreads * 32;
-constexpr int kKpt = 32;                     // keys per thread held in registers by the top-k
-constexpr int kRegKeys = kKpt * kThreads;    // 8192 pages; longer rows take the memory path
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
 #pragma unroll
@@ -54,77 +51,158 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
 }
 
 // Top-k of u[0..n) by (value descending, index ascending); ids written ascending.
-// Requires 0 < k < n.  All kThreads threads of the CTA call it.  Thread t owns the
-// contiguous keys [t*per, (t+1)*per); REG keeps them in registers (n <= kRegKeys).
-template <bool REG>
-__device__ void block_topk(const float* __restrict__ u, int n, int k, int32_t* __restrict__ ids) {
-    __shared__ uint32_t s_cnt[2][kWarps];
-    __shared__ uint32_t s_wtot[kWarps][2];
+// Requires 0 < k < n.  All kThreads threads of the CTA call it.  `skeys` is shared
+// memory for kSmemKeys keys that nothing else uses during the call; `sh` is
+// kTopkSmemWords words of shared scratch.
+//
+// Keys are the order-preserving integer images of the scores, staged once in
+// shared memory (longer rows re-read the scores from L2 instead).  Warp w owns the
+// contiguous index block [w*per_warp, (w+1)*per_warp); inside it lane l visits
+// l, l+32, ...  The code runs once per problem, so every phase is a short rolled
+// loop (straight-line code that is executed once costs an instruction-cache miss
+// per line):
+//   1. block min / max of the keys: the leading bits on which they agree need no
+//      search (scores of one problem share sign and exponent almost always);
+//   2. radix select of the k-th largest key on the bits that do vary, 8 bits per
+//      pass, histogram in shared memory (the worst case, every key in one bin, is
+//      32 serialised updates per warp instruction: microseconds, not more); as soon
+//      as at most kRankMax candidates share the selected prefix they are gathered
+//      and ranked directly, which ends the search;
+//   3. ordered compaction: keys above the threshold, plus the first
+//      k - #above keys equal to it in index order, ballot-ranked per warp.
+constexpr int kRankMax = 64;
+constexpr int kTopkSmemWords = 256 /*hist*/ + kRankMax /*candidates*/ + 32 /*scalars*/;
+constexpr int kSmemKeys = (int)(kRingBytes / 4);
+
+__device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int k, int32_t* __restrict__ ids,
+                                        uint32_t* __restrict__ skeys, uint32_t* __restrict__ sh) {
+    uint32_t* hist = sh;
+    uint32_t* cbuf = sh + 256;
+    uint32_t* sc = sh + 256 + kRankMax;         // [0..7] warp mins, [8..15] warp maxs / totals, [16..] results
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = (n + kThreads - 1) / kThreads;
-    const int lo = min(n, tid * per), hi = min(n, lo + per);
-    uint32_t key[REG ? kKpt : 1];
-    if (REG) {
-#pragma unroll
-        for (int j = 0; j < kKpt; ++j) key[j] = (lo + j < hi) ? float_key(__ldcg(u + lo + j)) : 0u;
-    }
-    auto key_at = [&](int i) -> uint32_t { return float_key(__ldcg(u + i)); };
+    const int per_warp = ((n + kThreads - 1) / kThreads) * 32;
+    const int J = per_warp / 32;                 // keys per lane
+    const int base = warp * per_warp + lane;
+    const unsigned lt = (1u << lane) - 1u;
+    const bool staged = n <= kSmemKeys;
 
-    // k-th largest key, one bit per step: the largest value v with #(key >= v) >= k
-    uint32_t tau = 0;
+    if (staged) {                                // eight loads in flight per thread
 #pragma unroll 1
-    for (int bit = 31; bit >= 0; --bit) {
-        const uint32_t cand = tau | (1u << bit);
-        uint32_t c = 0;
-        if (REG) {
+        for (int i0 = tid; i0 < n; i0 += 8 * kThreads) {
+            float f[8];
 #pragma unroll
-            for (int j = 0; j < kKpt; ++j) c += key[j] >= cand;
-        } else {
-            for (int i = lo; i < hi; ++i) c += key_at(i) >= cand;
+            for (int e = 0; e < 8; ++e) f[e] = i0 + e * kThreads < n ? __ldcg(u + i0 + e * kThreads) : 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) if (i0 + e * kThreads < n) skeys[i0 + e * kThreads] = float_key(f[e]);
         }
-        c = __reduce_add_sync(0xFFFFFFFFu, c);
-        if (lane == 0) s_cnt[bit & 1][warp] = c;
-        __syncthreads();
-        uint32_t tot = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) tot += s_cnt[bit & 1][w];
-        if (tot >= (uint32_t)k) tau = cand;
     }
-
-    uint32_t gt = 0, eq = 0;
-    if (REG) {
-#pragma unroll
-        for (int j = 0; j < kKpt; ++j) { gt += key[j] > tau; eq += (lo + j < hi) && key[j] == tau; }
-    } else {
-        for (int i = lo; i < hi; ++i) { uint32_t x = key_at(i); gt += x > tau; eq += x == tau; }
-    }
-    const uint32_t gi = warp_incl_scan(gt, lane), ei = warp_incl_scan(eq, lane);
-    if (lane == 31) { s_wtot[warp][0] = gi; s_wtot[warp][1] = ei; }
     __syncthreads();
-    uint32_t gb = gi - gt, eb = ei - eq, g_all = 0;
+    // fn(key, index, in_range) for every slot of this lane; all lanes call it J times.
+    // Unrolled by four so the shared-memory reads of neighbouring slots overlap.
+    auto for_each = [&](auto&& fn) {
+#pragma unroll 4
+        for (int j = 0; j < J; ++j) {
+            const int i = base + j * 32;
+            uint32_t x = 0u;
+            if (i < n) x = staged ? skeys[i] : float_key(__ldcg(u + i));
+            fn(x, i, i < n);
+        }
+    };
+
+    // ---- 1. range of the keys ---------------------------------------------------------------
+    uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
+    for_each([&](uint32_t x, int, bool ok) { if (ok) { kmn = min(kmn, x); kmx = max(kmx, x); } });
+    kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
+    kmx = __reduce_max_sync(0xFFFFFFFFu, kmx);
+    if (lane == 0) { sc[warp] = kmn; sc[8 + warp] = kmx; }
+    __syncthreads();
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        if (w < warp) { gb += s_wtot[w][0]; eb += s_wtot[w][1]; }
-        g_all += s_wtot[w][0];
-    }
-    const uint32_t ties = (uint32_t)k - g_all;     // keys equal to tau still to take
-    uint32_t pos = gb + min(eb, ties);
-    if (REG) {
+    for (int w2 = 0; w2 < kWarps; ++w2) { kmn = min(kmn, sc[w2]); kmx = max(kmx, sc[8 + w2]); }
+
+    // ---- 2. k-th largest key -----------------------------------------------------------------
+    int bits_left = 32 - __clz(kmn ^ kmx);       // low bits that differ somewhere (0: all keys equal)
+    uint32_t fixed_mask = bits_left >= 32 ? 0u : ~((1u << bits_left) - 1u);
+    uint32_t fixed_val = kmx & fixed_mask;
+    uint32_t krem = (uint32_t)k, cand = (uint32_t)n;
+    uint32_t tau = kmx;
+    bool found = bits_left == 0;
+#pragma unroll 1
+    while (!found) {
+        __syncthreads();                          // previous readers of hist / scalars are done
+        if (cand <= (uint32_t)kRankMax) {
+            // gather the candidates and rank them directly
+            if (tid == 0) sc[16] = 0u;
+            __syncthreads();
+            for_each([&](uint32_t x, int, bool ok) {
+                if (ok && (x & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[16], 1u)] = x;
+            });
+            __syncthreads();
+            if ((uint32_t)tid < cand) {
+                const uint32_t x = cbuf[tid];
+                uint32_t g = 0, e = 0;
+#pragma unroll 4
+                for (uint32_t i = 0; i < cand; ++i) { const uint32_t y = cbuf[i]; g += y > x; e += y == x; }
+                if (g < krem && krem <= g + e) sc[17] = x;      // every thread that qualifies holds the same key
+            }
+            __syncthreads();
+            tau = sc[17];
+            break;
+        }
+        const int nb = bits_left < 8 ? bits_left : 8, shift = bits_left - nb;
+        const uint32_t dmask = (1u << nb) - 1u;
+        hist[tid] = 0u;                           // kThreads == 256 bins
+        __syncthreads();
+        for_each([&](uint32_t x, int, bool ok) {
+            if (ok && (x & fixed_mask) == fixed_val) atomicAdd(&hist[(x >> shift) & dmask], 1u);
+        });
+        __syncthreads();
+        if (warp == 0) {                          // bin holding the krem-th largest candidate
+            uint32_t c8[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < kKpt; ++j) {
-            if (lo + j < hi) {
-                if (key[j] > tau) ids[pos++] = lo + j;
-                else if (key[j] == tau) { if (eb < ties) ids[pos++] = lo + j; ++eb; }
+            for (int i = 0; i < 8; ++i) { c8[i] = hist[255 - 8 * lane - i]; sum += c8[i]; }
+            const uint32_t incl = warp_incl_scan(sum, lane), excl = incl - sum;
+            if (excl < krem && krem <= incl) {
+                uint32_t run = excl;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (run < krem && krem <= run + c8[i]) { sc[18] = 255 - 8 * lane - i; sc[19] = krem - run; sc[20] = c8[i]; }
+                    run += c8[i];
+                }
             }
         }
-    } else {
-        for (int i = lo; i < hi; ++i) {
-            const uint32_t x = key_at(i);
-            if (x > tau) ids[pos++] = i;
-            else if (x == tau) { if (eb < ties) ids[pos++] = i; ++eb; }
-        }
+        __syncthreads();
+        const uint32_t digit = sc[18];
+        krem = sc[19]; cand = sc[20];
+        fixed_mask |= dmask << shift;
+        fixed_val |= digit << shift;
+        bits_left = shift;
+        if (bits_left == 0) { tau = fixed_val; found = true; }
     }
-    __syncthreads();                               // shared scratch is reused by the next call
+
+    // ---- 3. ordered compaction ---------------------------------------------------------------
+    uint32_t gt = 0, eq = 0;
+    for_each([&](uint32_t x, int, bool ok) { gt += ok && x > tau; eq += ok && x == tau; });
+    gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+    eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+    __syncthreads();
+    if (lane == 0) { sc[warp] = gt; sc[8 + warp] = eq; }
+    __syncthreads();
+    uint32_t run_gt = 0, run_eq = 0, all_gt = 0;
+#pragma unroll
+    for (int w2 = 0; w2 < kWarps; ++w2) {
+        if (w2 < warp) { run_gt += sc[w2]; run_eq += sc[8 + w2]; }
+        all_gt += sc[w2];
+    }
+    const uint32_t ties = (uint32_t)k - all_gt;   // keys equal to tau still to take, lowest indices first
+    for_each([&](uint32_t x, int i, bool ok) {
+        const bool g = ok && x > tau, e = ok && x == tau;
+        const unsigned bg = __ballot_sync(0xFFFFFFFFu, g), be = __ballot_sync(0xFFFFFFFFu, e);
+        const uint32_t g_before = run_gt + __popc(bg & lt), e_before = run_eq + __popc(be & lt);
+        if (g) ids[g_before + min(e_before, ties)] = i;
+        else if (e && e_before < ties) ids[g_before + e_before] = i;
+        run_gt += __popc(bg); run_eq += __popc(be);
+    });
+    __syncthreads();                              // the scratch may be reused by the caller
 }
 
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
@@ -182,6 +260,7 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
     constexpr int kPagesPerUnit = kWarps * (kSplit ? 1 : 2);
 
     extern __shared__ uint32_t ring_mem[];
+    __shared__ uint32_t s_topk[kTopkSmemWords];
     __shared__ int s_last;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -289,8 +368,8 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
         if (s_last) {
             __threadfence();
             int32_t* ids = page_ids + (size_t)problem * max_pages;
-            if (np <= kRegKeys) block_topk<true>(scores + row0, np, k_pg, ids);
-            else                block_topk<false>(scores + row0, np, k_pg, ids);
+            // the copy ring is idle here (all copies have landed): it stages the keys
+            block_topk(scores + row0, np, k_pg, ids, ring_mem, s_topk);
             if (tid == 0) n_pages[problem] = k_pg;
         }
     }

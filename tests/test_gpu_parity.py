@@ -131,9 +131,11 @@ def test_empty_and_single_token_sequences():
     assert (g["out"][0] == 0).all() and torch.isinf(g["lse"][0]).all()
 
 
-def test_more_pages_than_the_register_topk_holds():
-    # > 8192 pages per problem takes the memory-resident top-k path
-    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=1, t_cache=16 * 8300 + 5, token_budget=16 * 300)
+@pytest.mark.parametrize("pages", [8300, 16500])
+def test_long_rows_of_pages(pages):
+    # 16500 pages per problem is more than the selection stages in shared memory:
+    # it then re-reads the scores instead
+    w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=1, t_cache=16 * pages + 5, token_budget=16 * 300)
     d = W.make_inputs(w, DEV)
     g = H.gpu_pipeline(w, d)
     o = H.oracle_pipeline(w, d)
