@@ -16,7 +16,8 @@
 // Lane 0 brings both in with two bulk asynchronous copies (cp.async.bulk, the 1-D
 // TMA path) that signal the stage's mbarrier; the copies for the next kStages-1
 // pages are in flight while the warp computes on the current one, which is what
-// hides HBM latency at 8 warps per SM.  The list entry, sequence length and value
+// hides HBM latency (3 stages at 8 warps per SM; 6 stages at 4 warps per SM when
+// the call is too small to fill a wave and per-warp latency is what counts).  The list entry, sequence length and value
 // offsets a copy needs are fetched 32 pages at a time, one page per lane.
 //
 // A dropped value group is never copied for its own sake and never read: the
@@ -45,15 +46,18 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kStages = 3;
+constexpr int kStagesWide = 3;                   // two CTAs per SM (full-size calls)
+constexpr int kStagesDeep = 6;                   // one CTA per SM (calls too small to fill a wave)
 constexpr int kMaxGq = 8;
 constexpr int kCtasPerSm = 2;
 constexpr int kMinPagesPerWarp = 4;
 constexpr int kMaxSlots = 16;                    // partials per problem the merging warp handles (lane = slot, <= 32)
 constexpr uint32_t kKeyBytes = kPage * kRowBytes;          // 4096
 constexpr uint32_t kStageBytes = 2 * kKeyBytes;            // keys + worst-case value span
-constexpr uint32_t kRingBytes = kWarps * kStages * kStageBytes;
-constexpr uint32_t kSmemBytes = kRingBytes + 64 /* zero row, padded */ + kWarps * kStages * 8 /* mbarriers */;
+__host__ __device__ constexpr uint32_t ring_bytes(int stages) { return kWarps * stages * kStageBytes; }
+__host__ __device__ constexpr uint32_t smem_bytes(int stages) {      // ring + zero row (padded) + mbarriers
+    return ring_bytes(stages) + 64 + kWarps * stages * 8;
+}
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // ---- PTX wrappers -----------------------------------------------------------------------
@@ -151,9 +155,10 @@ struct PageRef {
     uint32_t groups;     // packed groups of the page actually stored
 };
 
-template <int S, bool MMA>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+template <int S, bool MMA, int kStages>
+__global__ void __launch_bounds__(kThreads, kStages == kStagesWide ? kCtasPerSm : 1)
 decode_attn_kernel(const AttnArgs a) {
+    constexpr uint32_t kRingBytes = ring_bytes(kStages);
     constexpr int OPG = kOctets / S;             // 16-byte chunks per value group
     constexpr uint32_t kGroupBytes = OPG * 16;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -489,55 +494,71 @@ decode_attn_kernel(const AttnArgs a) {
         old = __shfl_sync(0xFFFFFFFFu, old, 0);
         if (old + (unsigned)covered != (unsigned)mp) return;
         __threadfence();
-        // (1) lane = slot: all (max, sum) pairs of the problem in one round of loads (indices
-        //     clamped, so nothing is conditional), then per head the global max, each slot's
-        //     weight 2^(m - M) and the total of the normaliser
+        // Heads are merged kHB at a time (head indices clamped, so no load is conditional):
+        // (1) lane = slot: the (max, sum) pairs in one round of loads, then per head the
+        //     global max, each slot's weight 2^(m - M) and the total of the normaliser;
+        // (2) weighted sums in slot order, kSB slots' loads in flight; a lane owns 4 channels.
+        constexpr int kHB = MMA ? 4 : 1, kSB = MMA ? 4 : 8;
         const int sl_mine = min(lane, n_slots - 1);
-        float2 ml[kMaxGq];
+#pragma unroll 1
+        for (int h0 = 0; h0 < a.Gq; h0 += kHB) {
+            float wgt[kHB], M[kHB], L[kHB];
+            float2 ml[kHB];
 #pragma unroll
-        for (int h = 0; h < kMaxGq; ++h)
-            ml[h] = __ldcg(reinterpret_cast<const float2*>(a.part_ml) + slot0 + (size_t)sl_mine * a.Gq + min(h, a.Gq - 1));
-        float wgt[kMaxGq], M[kMaxGq], L[kMaxGq];
+            for (int i = 0; i < kHB; ++i)
+                ml[i] = __ldcg(reinterpret_cast<const float2*>(a.part_ml) + slot0 + (size_t)sl_mine * a.Gq +
+                               min(h0 + i, a.Gq - 1));
 #pragma unroll
-        for (int h = 0; h < kMaxGq; ++h) {
-            const float m = lane < n_slots ? ml[h].x : -INFINITY;
-            float mx = m;
+            for (int i = 0; i < kHB; ++i) {
+                const float m = lane < n_slots ? ml[i].x : -INFINITY;
+                float mx = m;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
-            wgt[h] = (m == -INFINITY) ? 0.f : exp2f(m - mx);
-            float ls = lane < n_slots ? ml[h].y * wgt[h] : 0.f;
+                for (int d = 1; d < 32; d <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
+                wgt[i] = (m == -INFINITY) ? 0.f : exp2f(m - mx);
+                float ls = lane < n_slots ? ml[i].y * wgt[i] : 0.f;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, d);
-            M[h] = mx; L[h] = ls;
-        }
-        // (2) weighted sums in slot order; each lane owns 4 channels of every head
-        float4 o[kMaxGq];
-#pragma unroll
-        for (int h = 0; h < kMaxGq; ++h) o[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-        for (int sl = 0; sl < n_slots; ++sl) {
-#pragma unroll
-            for (int h = 0; h < kMaxGq; ++h) {
-                const size_t ps = slot0 + (size_t)sl * a.Gq + min(h, a.Gq - 1);
-                const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_acc + ps * kHeadDim) + lane);
-                const float sc = __shfl_sync(0xFFFFFFFFu, wgt[h], sl);
-                o[h].x = fmaf(v.x, sc, o[h].x); o[h].y = fmaf(v.y, sc, o[h].y);
-                o[h].z = fmaf(v.z, sc, o[h].z); o[h].w = fmaf(v.w, sc, o[h].w);
+                for (int d = 1; d < 32; d <<= 1) ls += __shfl_xor_sync(0xFFFFFFFFu, ls, d);
+                M[i] = mx; L[i] = ls;
             }
-        }
+            float4 o[kHB];
 #pragma unroll
-        for (int h = 0; h < kMaxGq; ++h) {
-            if (h >= a.Gq) continue;
-            const float inv = L[h] > 0.f ? 1.f / L[h] : 0.f;
-            reinterpret_cast<float4*>(a.out + (row_base + h) * kHeadDim)[lane] =
-                make_float4(o[h].x * inv, o[h].y * inv, o[h].z * inv, o[h].w * inv);
-            if (a.lse && lane == 0) a.lse[row_base + h] = L[h] > 0.f ? (M[h] + log2f(L[h])) * ln2 : -INFINITY;
+            for (int i = 0; i < kHB; ++i) o[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+            for (int sl0 = 0; sl0 < n_slots; sl0 += kSB) {
+                float4 v[kSB][kHB];
+#pragma unroll
+                for (int j = 0; j < kSB; ++j)
+#pragma unroll
+                    for (int i = 0; i < kHB; ++i) {
+                        const size_t ps = slot0 + (size_t)min(sl0 + j, n_slots - 1) * a.Gq + min(h0 + i, a.Gq - 1);
+                        v[j][i] = __ldcg(reinterpret_cast<const float4*>(a.part_acc + ps * kHeadDim) + lane);
+                    }
+#pragma unroll
+                for (int j = 0; j < kSB; ++j)
+#pragma unroll
+                    for (int i = 0; i < kHB; ++i) {
+                        float sc = __shfl_sync(0xFFFFFFFFu, wgt[i], (sl0 + j) & 31);
+                        if (sl0 + j >= n_slots) sc = 0.f;
+                        o[i].x = fmaf(v[j][i].x, sc, o[i].x); o[i].y = fmaf(v[j][i].y, sc, o[i].y);
+                        o[i].z = fmaf(v[j][i].z, sc, o[i].z); o[i].w = fmaf(v[j][i].w, sc, o[i].w);
+                    }
+            }
+#pragma unroll
+            for (int i = 0; i < kHB; ++i) {
+                const int h = h0 + i;
+                if (h >= a.Gq) continue;
+                const float inv = L[i] > 0.f ? 1.f / L[i] : 0.f;
+                reinterpret_cast<float4*>(a.out + (row_base + h) * kHeadDim)[lane] =
+                    make_float4(o[i].x * inv, o[i].y * inv, o[i].z * inv, o[i].w * inv);
+                if (a.lse && lane == 0) a.lse[row_base + h] = L[i] > 0.f ? (M[i] + log2f(L[i])) * ln2 : -INFINITY;
+            }
         }
     };
 
     // ---- main loop ----------------------------------------------------------------------------
-    InFlight f0 = issue(0), f1 = issue(1), f2 = issue(2);
-    static_assert(kStages == 3, "the in-flight FIFO is written out for three stages");
+    InFlight f[kStages];                          // f[0] = oldest page in flight, in stage s
+#pragma unroll
+    for (int i = 0; i < kStages; ++i) f[i] = issue(i);
 
     int p_cur = (int)(x_lo / mp);
     int slot_cur = (int)(x_lo - (long long)p_cur * mp);
@@ -547,7 +568,7 @@ decode_attn_kernel(const AttnArgs a) {
     int s = 0;
 #pragma unroll 1
     for (int n = 0; n < count; ++n) {
-        if (f0.nv > 0) {                          // uniform across the warp
+        if (f[0].nv > 0) {                        // uniform across the warp
             const uint32_t par = (phase >> s) & 1u;
             phase ^= 1u << s;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(bars + 8 * s, par))) {
@@ -555,23 +576,29 @@ decode_attn_kernel(const AttnArgs a) {
                 // one more bounded wait each so they do not land in a dead CTA's memory,
                 // and leave; the outputs this worker owes stay unwritten.
                 if (lane == 0) atomicExch(a.status, (int)STC_ERR_TIMEOUT);
-                const int s1 = s + 1 == kStages ? 0 : s + 1, s2 = s1 + 1 == kStages ? 0 : s1 + 1;
-                if (f1.nv > 0) mbar_wait(bars + 8 * s1, (phase >> s1) & 1u);
-                if (f2.nv > 0) mbar_wait(bars + 8 * s2, (phase >> s2) & 1u);
+                int s2 = s;
+#pragma unroll
+                for (int i = 1; i < kStages; ++i) {
+                    s2 = s2 + 1 == kStages ? 0 : s2 + 1;
+                    if (f[i].nv > 0) mbar_wait(bars + 8 * s2, (phase >> s2) & 1u);
+                }
                 return;
             }
-            compute(s, f0);
+            compute(s, f[0]);
         }
         __syncwarp();
-        f0 = f1; f1 = f2; f2 = issue(s);
+#pragma unroll
+        for (int i = 0; i + 1 < kStages; ++i) f[i] = f[i + 1];
+        f[kStages - 1] = issue(s);
         s = s + 1 == kStages ? 0 : s + 1;
-        if (++slot_cur == mp) {                   // problem boundary inside the range
-            finish(p_cur, mp - seg_begin_slot);
-            ++p_cur; slot_cur = 0; seg_begin_slot = 0;
+        ++slot_cur;
+        if (slot_cur == mp || n + 1 == count) {   // the range leaves this problem (one call site: finish is big)
+            finish(p_cur, slot_cur - seg_begin_slot);
+            if (slot_cur == mp) { ++p_cur; slot_cur = 0; }
+            seg_begin_slot = slot_cur;
             if (n + 1 < count) { load_q(p_cur); reset_state(); }
         }
     }
-    if (slot_cur != 0) finish(p_cur, slot_cur - seg_begin_slot);
 }
 
 // out = 0, lse = -inf for every head: the call has nothing to attend.
@@ -582,17 +609,6 @@ __global__ void attn_empty_kernel(float* __restrict__ out, float* __restrict__ l
 }
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
-
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
 
 }  // namespace
 
@@ -606,6 +622,8 @@ AttnPlan attn_plan(const Geom& g, int max_pages) {
     long long workers = (total + kMinPagesPerWarp - 1) / kMinPagesPerWarp;
     const long long wave = 148LL * kCtasPerSm * kWarps;
     if (workers > wave) workers = wave;
+    // a call that fits one CTA per SM runs there, with the deeper ring
+    if (workers > 148LL * kWarps && workers < 148LL * kWarps * 3 / 2) workers = 148LL * kWarps;
     const long long by_slots = (long long)(kMaxSlots - 1) * (g.problems < 1 ? 1 : g.problems);
     if (workers > by_slots) workers = by_slots;  // keeps ceil(workers / problems) + 1 <= kMaxSlots
     if (workers < 1) workers = 1;
@@ -664,24 +682,25 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
     cudaError_t e = cudaMemsetAsync(wsp, 0, 256 + (size_t)g.problems * 4, st);
     if (e != cudaSuccess) return e;
     const int n_cta = (p.n_workers + kWarps - 1) / kWarps;
-    (void)sm_count;
-    const bool mma = g.Gq > 1;
+    const bool mma = g.Gq > 1, deep = n_cta <= 148;
+#define STC_ATTN_LAUNCH(S_, MMA_, ST_)                                                                  \
+    do {                                                                                                \
+        cudaFuncSetAttribute(decode_attn_kernel<S_, MMA_, ST_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                             (int)smem_bytes(ST_));                                                     \
+        decode_attn_kernel<S_, MMA_, ST_><<<n_cta, kThreads, smem_bytes(ST_), st>>>(a);                 \
+    } while (0)
 #define STC_ATTN(S_)                                                                                    \
     case S_:                                                                                            \
-        if (mma) {                                                                                      \
-            cudaFuncSetAttribute(decode_attn_kernel<S_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                 (int)kSmemBytes);                                                      \
-            decode_attn_kernel<S_, true><<<n_cta, kThreads, kSmemBytes, st>>>(a);                       \
-        } else {                                                                                        \
-            cudaFuncSetAttribute(decode_attn_kernel<S_, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                 (int)kSmemBytes);                                                      \
-            decode_attn_kernel<S_, false><<<n_cta, kThreads, kSmemBytes, st>>>(a);                      \
-        }                                                                                               \
+        if (mma && deep) STC_ATTN_LAUNCH(S_, true, kStagesDeep);                                        \
+        else if (mma) STC_ATTN_LAUNCH(S_, true, kStagesWide);                                           \
+        else if (deep) STC_ATTN_LAUNCH(S_, false, kStagesDeep);                                         \
+        else STC_ATTN_LAUNCH(S_, false, kStagesWide);                                                   \
         break;
     switch (g.S) {
         STC_ATTN(4) STC_ATTN(8) STC_ATTN(16)
         default: return cudaErrorInvalidValue;
     }
+#undef STC_ATTN_LAUNCH
 #undef STC_ATTN
     return cudaGetLastError();
 }
