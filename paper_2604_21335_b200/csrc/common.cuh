@@ -58,9 +58,9 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr) {
 // Order-preserving map from fp32 bits to uint32 (larger float -> larger key);
 // -0 is folded onto +0 so the two compare equal.
 __device__ __forceinline__ uint32_t float_key(float f) {
-    uint32_t u = __float_as_uint(f);
-    if ((u << 1) == 0u) u = 0u;
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    const uint32_t u = __float_as_uint(f);
+    const uint32_t k = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);   // negative: ~u, else u | sign
+    return k + (k == 0x7FFFFFFFu);                                          // -0 (0x7FFFFFFF) joins +0 (0x80000000)
 }
 
 // ---- internal launchers (one per source file) -------------------------------

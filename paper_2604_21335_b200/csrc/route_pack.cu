@@ -92,21 +92,33 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*
     return base + incl - v;
 }
 
-// Scores of one token -> order-preserving keys; best = first maximum.
+// Raw scores of one token (S/4 16-byte loads, issued together).
 template <int S>
-__device__ __forceinline__ void load_keys(const float* __restrict__ row, uint32_t (&key)[S], int& best) {
+__device__ __forceinline__ void load_raw(const float* __restrict__ row, uint4 (&raw)[S / 4]) {
     const uint4* p = reinterpret_cast<const uint4*>(row);
 #pragma unroll
+    for (int i = 0; i < S / 4; ++i) raw[i] = __ldg(p + i);   // L1-allocating: the row's 16-byte pieces share sectors
+}
+// Scores of one token -> order-preserving keys; best = first maximum (tracked by
+// value, so no register array is indexed at run time).
+template <int S>
+__device__ __forceinline__ void make_keys(const uint4 (&raw)[S / 4], uint32_t (&key)[S], int& best) {
+#pragma unroll
     for (int i = 0; i < S / 4; ++i) {
-        uint4 w = ldg_nc16(p + i);
+        const uint4 w = raw[i];
         key[4 * i + 0] = float_key(__uint_as_float(w.x));
         key[4 * i + 1] = float_key(__uint_as_float(w.y));
         key[4 * i + 2] = float_key(__uint_as_float(w.z));
         key[4 * i + 3] = float_key(__uint_as_float(w.w));
     }
+    uint32_t bk = key[0];
     best = 0;
 #pragma unroll
-    for (int j = 1; j < S; ++j) if (key[j] > key[best]) best = j;
+    for (int j = 1; j < S; ++j) {
+        const bool up = key[j] > bk;
+        bk = up ? key[j] : bk;
+        best = up ? j : best;
+    }
 }
 
 __device__ __forceinline__ int token_class(const uint8_t* cls, int t, int len) {
@@ -145,14 +157,15 @@ template <int S>
 __global__ void __launch_bounds__(kThreads)
 route_hist_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
                   int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int n_tiles,
-                  int k_nominal, int min_per_token, int pass, uint32_t* __restrict__ state_all,
-                  uint32_t* __restrict__ hist_all) {
+                  int tiles_per_cta, int k_nominal, int min_per_token, int pass,
+                  uint32_t* __restrict__ state_all, uint32_t* __restrict__ hist_all) {
     __shared__ uint32_t shist[kBins];
     __shared__ uint32_t s_w[kWarps];
     __shared__ uint32_t s_pick[2];
     __shared__ int s_last;
 
-    const int problem = blockIdx.x / n_tiles, tile = blockIdx.x - problem * n_tiles;
+    const int n_groups = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    const int problem = blockIdx.x / n_groups, group = blockIdx.x - problem * n_groups;
     const int b = problem / Hkv, hk = problem - b * Hkv;
     const int len = clamp_len(seq_len, b, T);
     uint32_t* state = state_all + (size_t)problem * ST_WORDS;
@@ -165,23 +178,38 @@ route_hist_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
         prefix = __ldcg(state + ST_PREFIX);
     }
     const uint32_t himask = pass_himask(pass);
+    const int dshift = pass_shift(pass);
+    const uint32_t dmask = pass == 2 ? 1023u : 2047u;
     for (int i = tid; i < kBins; i += kThreads) shist[i] = 0;
     __syncthreads();
 
     const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
     uint32_t n_routed = 0;
+    // several 1024-token tiles per CTA: the shared histogram is cleared and flushed once
+    const int tile_end = min(n_tiles, (group + 1) * tiles_per_cta);
+#pragma unroll 1
+    for (int tile = group * tiles_per_cta; tile < tile_end; ++tile) {
+        if (tile * kTile >= len) break;
+        uint4 raw[kTokPerThread][S / 4];          // all of the thread's loads are in flight before the first use
+        bool routed[kTokPerThread];
 #pragma unroll
-    for (int i = 0; i < kTokPerThread; ++i) {
-        const int t = tile * kTile + i * kThreads + tid;
-        if (token_class(c, t, len) != STC_CLS_ROUTED) continue;
-        ++n_routed;
-        uint32_t key[S];
-        int best;
-        load_keys<S>(scores + ((size_t)problem * T + t) * S, key, best);
+        for (int i = 0; i < kTokPerThread; ++i) {
+            const int t = tile * kTile + i * kThreads + tid;
+            routed[i] = token_class(c, t, len) == STC_CLS_ROUTED;
+            if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+        }
 #pragma unroll
-        for (int j = 0; j < S; ++j) {
-            if (min_per_token && j == best) continue;
-            if ((key[j] & himask) == prefix) atomicAdd(&shist[pass_digit(key[j], pass)], 1u);
+        for (int i = 0; i < kTokPerThread; ++i) {
+            if (!routed[i]) continue;
+            ++n_routed;
+            uint32_t key[S];
+            int best;
+            make_keys<S>(raw[i], key, best);
+#pragma unroll
+            const int skip = min_per_token ? best : -1;
+#pragma unroll
+            for (int j = 0; j < S; ++j)
+                if (j != skip && (key[j] & himask) == prefix) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
         }
     }
     __syncthreads();
@@ -197,7 +225,7 @@ route_hist_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
 
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(state + ST_TICKET0 + pass, 1u) == (unsigned)(n_tiles - 1));
+    if (tid == 0) s_last = (atomicAdd(state + ST_TICKET0 + pass, 1u) == (unsigned)(n_groups - 1));
     __syncthreads();
     if (!s_last) return;
     __threadfence();
@@ -229,11 +257,12 @@ template <int S>
 __global__ void __launch_bounds__(kThreads)
 route_mask_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
                   int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int n_tiles,
-                  int k_nominal, int min_per_token, int mode, const uint32_t* __restrict__ state_all,
-                  uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
-                  uint32_t* __restrict__ tile_sums) {
+                  int tiles_per_cta, int k_nominal, int min_per_token, int mode,
+                  const uint32_t* __restrict__ state_all, uint16_t* __restrict__ v_mask,
+                  uint16_t* __restrict__ tie_all, uint32_t* __restrict__ tile_sums) {
     __shared__ uint32_t s_w[kWarps];
-    const int problem = blockIdx.x / n_tiles, tile = blockIdx.x - problem * n_tiles;
+    const int n_groups = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
+    const int problem = blockIdx.x / n_groups, group = blockIdx.x - problem * n_groups;
     const int b = problem / Hkv, hk = problem - b * Hkv;
     const int len = clamp_len(seq_len, b, T);
     const int tid = threadIdx.x;
@@ -245,12 +274,24 @@ route_mask_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
         flags = __ldcg(state + ST_FLAGS);
         tau = __ldcg(state + ST_PREFIX);
     }
+    const int tile_end = min(n_tiles, (group + 1) * tiles_per_cta);
+#pragma unroll 1
+    for (int tile = group * tiles_per_cta; tile < tile_end; ++tile) {
     uint32_t n_def = 0, n_tie = 0;
+    uint4 raw[kTokPerThread][S / 4];              // loads first, arithmetic after
+    int cls_of[kTokPerThread];
+#pragma unroll
+    for (int i = 0; i < kTokPerThread; ++i) {
+        const int t = tile * kTile + i * kThreads + tid;
+        cls_of[i] = t < T ? token_class(c, t, len) : STC_CLS_DROP;
+        if (cls_of[i] == STC_CLS_ROUTED && !(flags & FL_BUDGET))
+            load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+    }
 #pragma unroll
     for (int i = 0; i < kTokPerThread; ++i) {
         const int t = tile * kTile + i * kThreads + tid;
         if (t >= T) continue;
-        const int cl = token_class(c, t, len);
+        const int cl = cls_of[i];
         uint32_t def = 0, tie = 0;
         if (flags & FL_BUDGET) {
             def = 0;
@@ -259,7 +300,7 @@ route_mask_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
         } else if (cl == STC_CLS_ROUTED) {
             uint32_t key[S];
             int best;
-            load_keys<S>(scores + ((size_t)problem * T + t) * S, key, best);
+            make_keys<S>(raw[i], key, best);
             if (mode == STC_MODE_PER_TOKEN) {
 #pragma unroll
                 for (int j = 0; j < S; ++j) {
@@ -290,6 +331,7 @@ route_mask_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
     if (tid == 0) {
         tile_sums[((size_t)problem * n_tiles + tile) * 2 + 0] = tot_def;
         tile_sums[((size_t)problem * n_tiles + tile) * 2 + 1] = tot_tie;
+    }
     }
 }
 
@@ -415,6 +457,10 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     const int n_tiles = (g.T + kTile - 1) / kTile;
     const long long n_cta = (long long)n_tiles * g.problems;
     if (n_cta > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    // score-scanning kernels: enough CTAs for a few waves, several tiles each beyond that
+    int tpc = (int)(n_cta / (148 * 8 * 2));
+    tpc = tpc < 1 ? 1 : (tpc > 16 ? 16 : tpc);
+    const unsigned n_cta_scan = (unsigned)((n_tiles + tpc - 1) / tpc) * (unsigned)g.problems;
     const int64_t cls_h = class_head_stride;
     const int64_t cls_b = class_head_stride ? (int64_t)g.Hkv * class_head_stride : (int64_t)g.T;
     cudaError_t e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
@@ -424,11 +470,11 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     case S_: {                                                                                      \
         if (mode == STC_MODE_GLOBAL)                                                                \
             for (int pass = 0; pass < 3; ++pass)                                                    \
-                route_hist_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                        \
-                    scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, k_nominal,     \
+                route_hist_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                             \
+                    scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal, \
                     min_per_token, pass, w.state, w.hist);                                          \
-        route_mask_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                                \
-            scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, k_nominal,             \
+        route_mask_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                                     \
+            scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal,        \
             min_per_token, mode, w.state, v_mask, w.tie, w.tile_sums);                              \
         route_compact_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                             \
             static_cast<const uint4*>(v), g.seq_len, g.Hkv, g.T, n_tiles, mode, w.state,            \
