@@ -38,7 +38,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kCtasPerSm = 2;
-constexpr int kDepth = 8;                    // units in flight per lane (32 B each)
+constexpr int kDepth = 8;                    // (a power of two)                    // units in flight per lane (32 B each)
 constexpr size_t kRingBytes = (size_t)kDepth * kThreads * 32;
 
 __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
@@ -71,14 +71,14 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
 //   3. ordered compaction: keys above the threshold, plus the first
 //      k - #above keys equal to it in index order, ballot-ranked per warp.
 constexpr int kRankMax = 64;
-constexpr int kTopkSmemWords = 256 /*hist*/ + kRankMax /*candidates*/ + 32 /*scalars*/;
+constexpr int kTopkSmemWords = 256 /*hist*/ + kRankMax /*candidates*/ + 2 * kWarps + 8 /*scalars*/;
 constexpr int kSmemKeys = (int)(kRingBytes / 4);
 
 __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int k, int32_t* __restrict__ ids,
                                         uint32_t* __restrict__ skeys, uint32_t* __restrict__ sh) {
     uint32_t* hist = sh;
     uint32_t* cbuf = sh + 256;
-    uint32_t* sc = sh + 256 + kRankMax;         // [0..7] warp mins, [8..15] warp maxs / totals, [16..] results
+    uint32_t* sc = sh + 256 + kRankMax;         // [kWarps] warp mins, [kWarps] warp maxs / totals, then results
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int per_warp = ((n + kThreads - 1) / kThreads) * 32;
     const int J = per_warp / 32;                 // keys per lane
@@ -114,10 +114,10 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
     for_each([&](uint32_t x, int, bool ok) { if (ok) { kmn = min(kmn, x); kmx = max(kmx, x); } });
     kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
     kmx = __reduce_max_sync(0xFFFFFFFFu, kmx);
-    if (lane == 0) { sc[warp] = kmn; sc[8 + warp] = kmx; }
+    if (lane == 0) { sc[warp] = kmn; sc[kWarps + warp] = kmx; }
     __syncthreads();
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) { kmn = min(kmn, sc[w2]); kmx = max(kmx, sc[8 + w2]); }
+    for (int w2 = 0; w2 < kWarps; ++w2) { kmn = min(kmn, sc[w2]); kmx = max(kmx, sc[kWarps + w2]); }
 
     // ---- 2. k-th largest key -----------------------------------------------------------------
     int bits_left = 32 - __clz(kmn ^ kmx);       // low bits that differ somewhere (0: all keys equal)
@@ -131,10 +131,10 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
         __syncthreads();                          // previous readers of hist / scalars are done
         if (cand <= (uint32_t)kRankMax) {
             // gather the candidates and rank them directly
-            if (tid == 0) sc[16] = 0u;
+            if (tid == 0) sc[2 * kWarps] = 0u;
             __syncthreads();
             for_each([&](uint32_t x, int, bool ok) {
-                if (ok && (x & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[16], 1u)] = x;
+                if (ok && (x & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[2 * kWarps], 1u)] = x;
             });
             __syncthreads();
             if ((uint32_t)tid < cand) {
@@ -142,15 +142,15 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
                 uint32_t g = 0, e = 0;
 #pragma unroll 4
                 for (uint32_t i = 0; i < cand; ++i) { const uint32_t y = cbuf[i]; g += y > x; e += y == x; }
-                if (g < krem && krem <= g + e) sc[17] = x;      // every thread that qualifies holds the same key
+                if (g < krem && krem <= g + e) sc[2 * kWarps + 1] = x;      // every thread that qualifies holds the same key
             }
             __syncthreads();
-            tau = sc[17];
+            tau = sc[2 * kWarps + 1];
             break;
         }
         const int nb = bits_left < 8 ? bits_left : 8, shift = bits_left - nb;
         const uint32_t dmask = (1u << nb) - 1u;
-        hist[tid] = 0u;                           // kThreads == 256 bins
+        if (tid < 256) hist[tid] = 0u;
         __syncthreads();
         for_each([&](uint32_t x, int, bool ok) {
             if (ok && (x & fixed_mask) == fixed_val) atomicAdd(&hist[(x >> shift) & dmask], 1u);
@@ -165,14 +165,14 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
                 uint32_t run = excl;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    if (run < krem && krem <= run + c8[i]) { sc[18] = 255 - 8 * lane - i; sc[19] = krem - run; sc[20] = c8[i]; }
+                    if (run < krem && krem <= run + c8[i]) { sc[2 * kWarps + 2] = 255 - 8 * lane - i; sc[2 * kWarps + 3] = krem - run; sc[2 * kWarps + 4] = c8[i]; }
                     run += c8[i];
                 }
             }
         }
         __syncthreads();
-        const uint32_t digit = sc[18];
-        krem = sc[19]; cand = sc[20];
+        const uint32_t digit = sc[2 * kWarps + 2];
+        krem = sc[2 * kWarps + 3]; cand = sc[2 * kWarps + 4];
         fixed_mask |= dmask << shift;
         fixed_val |= digit << shift;
         bits_left = shift;
@@ -185,12 +185,12 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
     gt = __reduce_add_sync(0xFFFFFFFFu, gt);
     eq = __reduce_add_sync(0xFFFFFFFFu, eq);
     __syncthreads();
-    if (lane == 0) { sc[warp] = gt; sc[8 + warp] = eq; }
+    if (lane == 0) { sc[warp] = gt; sc[kWarps + warp] = eq; }
     __syncthreads();
     uint32_t run_gt = 0, run_eq = 0, all_gt = 0;
 #pragma unroll
     for (int w2 = 0; w2 < kWarps; ++w2) {
-        if (w2 < warp) { run_gt += sc[w2]; run_eq += sc[8 + w2]; }
+        if (w2 < warp) { run_gt += sc[w2]; run_eq += sc[kWarps + w2]; }
         all_gt += sc[w2];
     }
     const uint32_t ties = (uint32_t)k - all_gt;   // keys equal to tau still to take, lowest indices first
@@ -294,16 +294,26 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
         if (trivial && !scores_wanted) continue;
 
         const size_t row0 = (size_t)problem * P;
+        // units of the segment in which this half-warp's page exists (pages advance by
+        // kPagesPerUnit per unit, so validity is a prefix of the units)
+        const int page0 = u_begin * kPagesPerUnit + sub;
+        const int lim = max(0, min(n, (np - page0 + kPagesPerUnit - 1) / kPagesPerUnit));
+        // running source pointers / ring slot of the next unit to issue (units are issued in order)
+        const uint4* src_min = kmin + (row0 + page0) * kOctets + l;
+        const uint4* src_max = kmax + (row0 + page0) * kOctets + l;
+        uint32_t slot_off = 0;
         auto issue = [&](int i) {                 // unit i of the segment -> slot i % kDepth
-            const int page = (u_begin + i) * kPagesPerUnit + sub;
-            if (i < n && page < np) {
-                const uint32_t dst = ring + (uint32_t)(i % kDepth) * kSlotBytes;
-                const size_t src = (row0 + page) * kOctets + l;
-                cp_async16(dst, kmin + src);
-                cp_async16(dst + 512u, kmax + src);
+            if (i < lim) {
+                cp_async16(ring + slot_off, src_min);
+                cp_async16(ring + slot_off + 512u, src_max);
             }
             cp_async_commit();
+            src_min += kPagesPerUnit * kOctets;
+            src_max += kPagesPerUnit * kOctets;
+            slot_off = (slot_off + kSlotBytes) & (kDepth * kSlotBytes - 1u);
         };
+        float* dst_score = scores + row0 + page0;
+        const bool writer = l == 0 && (!kSplit || half == 0);
 #pragma unroll
         for (int i = 0; i < kDepth; ++i) issue(i);
 
@@ -321,7 +331,6 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             }
         }
         auto score_unit = [&](int i, const uint4& lo, const uint4& hi) {
-            const int page = (u_begin + i) * kPagesPerUnit + sub;
             const uint32_t wl[4] = {lo.x, lo.y, lo.z, lo.w}, wh[4] = {hi.x, hi.y, hi.z, hi.w};
             uint64_t a2[4], z2[4];
 #pragma unroll
@@ -339,14 +348,15 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             }
             float best = reduce_heads<NH>(v, l, hm);
             if (kSplit) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, 16));
-            if (l == 0 && (!kSplit || half == 0) && i < n && page < np) scores[row0 + page] = best;
+            if (writer && i < lim) *dst_score = best;
+            dst_score += kPagesPerUnit;
         };
 
 #pragma unroll 1
         for (int i = 0; i < n; i += 2) {
             cp_async_wait<kDepth - 2>();           // units i and i+1 have landed
-            const uint32_t s0 = ring + (uint32_t)(i % kDepth) * kSlotBytes;
-            const uint32_t s1 = ring + (uint32_t)((i + 1) % kDepth) * kSlotBytes;
+            const uint32_t s0 = ring + (uint32_t)(i & (kDepth - 1)) * kSlotBytes;
+            const uint32_t s1 = ring + (uint32_t)((i + 1) & (kDepth - 1)) * kSlotBytes;
             const uint4 lo0 = lds16(s0), hi0 = lds16(s0 + 512u);
             const uint4 lo1 = lds16(s1), hi1 = lds16(s1 + 512u);
             score_unit(i, lo0, hi0);
