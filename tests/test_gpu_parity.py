@@ -57,6 +57,16 @@ def test_shrunken_configs(name, over, seq):
     full_parity(w, seq_len=seq)
 
 
+@pytest.mark.parametrize("budget", W.CFG4_BUDGETS)
+@pytest.mark.parametrize("keep", W.CFG4_KEEPS)
+def test_cfg4_sweep_points_shrunken(budget, keep):
+    """Every (token budget, keep ratio) point of the long-context sweep on a shorter context."""
+    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=8, n_kv_heads=2, t_cache=16 * 1100 + 9,
+                 token_budget=budget, k_nominal=keep)
+    d, g, o, _ = full_parity(w, seq_len=[w.t_cache, 16 * 700 + 3])
+    assert (o["n_pages"] == budget // 16).all()
+
+
 def test_cfg3_class_layout_and_totals():
     w = W.shrink(W.get("cfg3"), batch=2, n_q_heads=8, n_kv_heads=8)
     d, g, o, _ = full_parity(w)
@@ -204,8 +214,16 @@ def _problem_slice(w, d, b, hk):
     return w1, d1
 
 
+def test_cfg3_full_size_whole_batch():
+    """The VLM-shaped cache at its benchmarked size: every problem against the checker."""
+    w = W.get("cfg3")
+    d, g, o, _ = full_parity(w)
+    assert o["page_ids"] is None and (o["total"] == 128 * 8 + 144 * 3).all()
+
+
 @pytest.mark.parametrize("name,samples", [("cfg1", [(0, 0), (0, 13), (0, 31)]),
-                                          ("cfg2", [(0, 0), (5, 2), (7, 3)])])
+                                          ("cfg2", [(0, 0), (5, 2), (7, 3)]),
+                                          ("cfg4", [(0, 0), (9, 5)])])
 def test_full_size_sampled_problems(name, samples):
     """At the benchmarked sizes: whole pass on the GPU, sampled problems on the checker."""
     w = W.get(name)
