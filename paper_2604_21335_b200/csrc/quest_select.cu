@@ -80,38 +80,72 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
     uint32_t* cbuf = sh + 256;
     uint32_t* sc = sh + 256 + kRankMax;         // [kWarps] warp mins, [kWarps] warp maxs / totals, then results
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per_warp = ((n + kThreads - 1) / kThreads) * 32;
-    const int J = per_warp / 32;                 // keys per lane
-    const int base = warp * per_warp + lane;
+    // Warp w owns the index block [w*per_warp, (w+1)*per_warp); a lane visits groups of four
+    // consecutive keys (one 16-byte read), group j*32 + lane in pass j.  Slots past n hold key 0,
+    // which is below every real key, so it can never be selected (k < n).
+    const int per_warp = ((n + kWarps * 128 - 1) / (kWarps * 128)) * 128;
+    const int J = per_warp / 128;                // groups per lane
+    const int padded = per_warp * kWarps;
     const unsigned lt = (1u << lane) - 1u;
-    const bool staged = n <= kSmemKeys;
+    const bool staged = padded <= kSmemKeys;
 
-    if (staged) {                                // eight loads in flight per thread
+    // ---- 1. stage the keys, block min / max on the way ----------------------------------------
+    uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
+    if (staged) {
+        // up to eight groups per thread in flight (one round trip to L2 for 8192 keys)
+        const bool vec = (reinterpret_cast<uintptr_t>(u) & 15u) == 0;
 #pragma unroll 1
-        for (int i0 = tid; i0 < n; i0 += 8 * kThreads) {
-            float f[8];
+        for (int g0 = tid; g0 < padded / 4; g0 += 8 * kThreads) {
+            uint4 raw[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = i0 + e * kThreads < n ? __ldcg(u + i0 + e * kThreads) : 0.f;
+            for (int e = 0; e < 8; ++e) {
+                const int i = 4 * (g0 + e * kThreads);
+                raw[e] = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);   // -NaN: key 0
+                if (vec && i + 3 < n) {
+                    raw[e] = __ldcg(reinterpret_cast<const uint4*>(u + i));
+                } else {
+                    if (i < n) raw[e].x = __float_as_uint(__ldcg(u + i));
+                    if (i + 1 < n) raw[e].y = __float_as_uint(__ldcg(u + i + 1));
+                    if (i + 2 < n) raw[e].z = __float_as_uint(__ldcg(u + i + 2));
+                    if (i + 3 < n) raw[e].w = __float_as_uint(__ldcg(u + i + 3));
+                }
+            }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) if (i0 + e * kThreads < n) skeys[i0 + e * kThreads] = float_key(f[e]);
+            for (int e = 0; e < 8; ++e) {
+                const int i = 4 * (g0 + e * kThreads);
+                if (i >= padded) continue;
+                const uint32_t w4[4] = {raw[e].x, raw[e].y, raw[e].z, raw[e].w};
+                uint32_t x[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    x[c] = i + c < n ? float_key(__uint_as_float(w4[c])) : 0u;
+                    if (i + c < n) { kmn = min(kmn, x[c]); kmx = max(kmx, x[c]); }
+                }
+                *reinterpret_cast<uint4*>(skeys + i) = make_uint4(x[0], x[1], x[2], x[3]);
+            }
         }
     }
-    __syncthreads();
-    // fn(key, index, in_range) for every slot of this lane; all lanes call it J times.
-    // Unrolled by four so the shared-memory reads of neighbouring slots overlap.
+    // fn(keys[4], first index) for every group of this lane; all lanes call it J times
     auto for_each = [&](auto&& fn) {
-#pragma unroll 4
+#pragma unroll 2
         for (int j = 0; j < J; ++j) {
-            const int i = base + j * 32;
-            uint32_t x = 0u;
-            if (i < n) x = staged ? skeys[i] : float_key(__ldcg(u + i));
-            fn(x, i, i < n);
+            const int i0 = warp * per_warp + (j * 32 + lane) * 4;
+            uint32_t x[4];
+            if (staged) {
+                const uint4 v = *reinterpret_cast<const uint4*>(skeys + i0);
+                x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) x[e] = i0 + e < n ? float_key(__ldcg(u + i0 + e)) : 0u;
+            }
+            fn(x, i0);
         }
     };
-
-    // ---- 1. range of the keys ---------------------------------------------------------------
-    uint32_t kmn = 0xFFFFFFFFu, kmx = 0u;
-    for_each([&](uint32_t x, int, bool ok) { if (ok) { kmn = min(kmn, x); kmx = max(kmx, x); } });
+    if (!staged)
+        for_each([&](const uint32_t (&x)[4], int i0) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) if (i0 + e < n) { kmn = min(kmn, x[e]); kmx = max(kmx, x[e]); }
+        });
     kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
     kmx = __reduce_max_sync(0xFFFFFFFFu, kmx);
     if (lane == 0) { sc[warp] = kmn; sc[kWarps + warp] = kmx; }
@@ -133,8 +167,10 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
             // gather the candidates and rank them directly
             if (tid == 0) sc[2 * kWarps] = 0u;
             __syncthreads();
-            for_each([&](uint32_t x, int, bool ok) {
-                if (ok && (x & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[2 * kWarps], 1u)] = x;
+            for_each([&](const uint32_t (&x)[4], int) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (x[e] != 0u && (x[e] & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[2 * kWarps], 1u)] = x[e];
             });
             __syncthreads();
             if ((uint32_t)tid < cand) {
@@ -142,7 +178,7 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
                 uint32_t g = 0, e = 0;
 #pragma unroll 4
                 for (uint32_t i = 0; i < cand; ++i) { const uint32_t y = cbuf[i]; g += y > x; e += y == x; }
-                if (g < krem && krem <= g + e) sc[2 * kWarps + 1] = x;      // every thread that qualifies holds the same key
+                if (g < krem && krem <= g + e) sc[2 * kWarps + 1] = x;   // every thread that qualifies holds the same key
             }
             __syncthreads();
             tau = sc[2 * kWarps + 1];
@@ -152,8 +188,10 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
         const uint32_t dmask = (1u << nb) - 1u;
         if (tid < 256) hist[tid] = 0u;
         __syncthreads();
-        for_each([&](uint32_t x, int, bool ok) {
-            if (ok && (x & fixed_mask) == fixed_val) atomicAdd(&hist[(x >> shift) & dmask], 1u);
+        for_each([&](const uint32_t (&x)[4], int) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (x[e] != 0u && (x[e] & fixed_mask) == fixed_val) atomicAdd(&hist[(x[e] >> shift) & dmask], 1u);
         });
         __syncthreads();
         if (warp == 0) {                          // bin holding the krem-th largest candidate
@@ -165,7 +203,9 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
                 uint32_t run = excl;
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    if (run < krem && krem <= run + c8[i]) { sc[2 * kWarps + 2] = 255 - 8 * lane - i; sc[2 * kWarps + 3] = krem - run; sc[2 * kWarps + 4] = c8[i]; }
+                    if (run < krem && krem <= run + c8[i]) {
+                        sc[2 * kWarps + 2] = 255 - 8 * lane - i; sc[2 * kWarps + 3] = krem - run; sc[2 * kWarps + 4] = c8[i];
+                    }
                     run += c8[i];
                 }
             }
@@ -180,8 +220,12 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
     }
 
     // ---- 3. ordered compaction ---------------------------------------------------------------
+    // counts packed as (#above) | (#equal) << 16 : a warp holds at most 4096 keys per pass
     uint32_t gt = 0, eq = 0;
-    for_each([&](uint32_t x, int, bool ok) { gt += ok && x > tau; eq += ok && x == tau; });
+    for_each([&](const uint32_t (&x)[4], int) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { gt += x[e] > tau; eq += x[e] == tau; }
+    });
     gt = __reduce_add_sync(0xFFFFFFFFu, gt);
     eq = __reduce_add_sync(0xFFFFFFFFu, eq);
     __syncthreads();
@@ -194,13 +238,19 @@ __device__ __noinline__ void block_topk(const float* __restrict__ u, int n, int 
         all_gt += sc[w2];
     }
     const uint32_t ties = (uint32_t)k - all_gt;   // keys equal to tau still to take, lowest indices first
-    for_each([&](uint32_t x, int i, bool ok) {
-        const bool g = ok && x > tau, e = ok && x == tau;
-        const unsigned bg = __ballot_sync(0xFFFFFFFFu, g), be = __ballot_sync(0xFFFFFFFFu, e);
-        const uint32_t g_before = run_gt + __popc(bg & lt), e_before = run_eq + __popc(be & lt);
-        if (g) ids[g_before + min(e_before, ties)] = i;
-        else if (e && e_before < ties) ids[g_before + e_before] = i;
-        run_gt += __popc(bg); run_eq += __popc(be);
+    for_each([&](const uint32_t (&x)[4], int i0) {
+        uint32_t mine = 0;                        // this lane's four keys: #above | #equal << 16
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mine += (x[e] > tau) + ((uint32_t)(x[e] == tau) << 16);
+        const uint32_t incl = warp_incl_scan(mine, lane), before = incl - mine;
+        uint32_t g_before = run_gt + (before & 0xFFFFu), e_before = run_eq + (before >> 16);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (x[e] > tau) { ids[g_before + min(e_before, ties)] = i0 + e; ++g_before; }
+            else if (x[e] == tau) { if (e_before < ties) ids[g_before + e_before] = i0 + e; ++e_before; }
+        }
+        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        run_gt += tot & 0xFFFFu; run_eq += tot >> 16;
     });
     __syncthreads();                              // the scratch may be reused by the caller
 }
@@ -259,7 +309,7 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
     constexpr int NH = kSplit ? 4 : (GQ == 3 ? 4 : GQ);   // heads per lane, padded to 1 / 2 / 4
     constexpr int kPagesPerUnit = kWarps * (kSplit ? 1 : 2);
 
-    extern __shared__ uint32_t ring_mem[];
+    extern __shared__ __align__(16) uint32_t ring_mem[];
     __shared__ uint32_t s_topk[kTopkSmemWords];
     __shared__ int s_last;
 
