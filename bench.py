@@ -52,14 +52,14 @@ def algorithmic_bytes(w: W.Workload, seq_len, n_routed, n_full, total_groups, se
     meta = tok * 256 + pages * 512
     route = (n_routed * w.n_groups * 4                         # router scores, once
              + (tok if w.n_text else 0)                         # token classes
-             + total_groups * g2 * 2                            # kept groups in + out
-             + tok * 2 + (tok + w.n_problems) * 4)              # masks + offsets
+             + tok * 2)                                         # masks
+    pack = total_groups * g2 * 2 + (tok + w.n_problems) * 4    # kept groups in + out, offsets
     q_out = w.batch * Hq * (256 + 512)
     select = 0
     if w.token_budget is not None:
         select = pages * 512 + w.batch * Hq * 256 + sel_pages * 4 + w.n_problems * 4
     attn = sel_tokens * 256 + sel_groups * g2 + sel_tokens * 2 + sel_pages * 8 + q_out
-    return dict(page_meta=meta, route_pack=route, quest_select=select, decode_attn=attn)
+    return dict(page_meta=meta, route_mask=route, pack_values=pack, quest_select=select, decode_attn=attn)
 
 
 def peaks() -> tuple[float, str]:
@@ -218,15 +218,16 @@ def run_gpu(args, r: D.Rank):
     ws_s = Bd.new_workspace(shape, Bd.OP_QUEST_SELECT, device=dev)
     ws_a = Bd.new_workspace(shape, Bd.OP_DECODE_ATTN, max_pages, device=dev)
     qs = [d["q"][i].contiguous() for i in range(NQ)]
-    names = ["page_meta", "route_pack", "quest_select", "decode_attn"]
-    launches_per_step = 1 + (5 if True else 2) + (1 if page_ids is not None else 0) + 1
+    names = ["page_meta", "route_mask", "pack_values", "quest_select", "decode_attn"]
+    launches_per_step = 1 + 5 + (1 if page_ids is not None else 0) + 1   # route_mask = 3 histogram passes + mask
 
     def step(i, ev=None):
         q = qs[i % NQ]
         if ev: ev[0].record()
         P.build_page_meta(shape, cache)
         if ev: ev[1].record()
-        P.route_pack(shape, d["v"], d["scores"], d["tok_class"], w.k_nominal, cache, total, status, ws_r)
+        P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)     # stc_route_pack, first half
+        P.pack_values(shape, d["v"], cache, total, status, ws_r)                       # ... second half
         if ev: ev[2].record()
         if page_ids is not None:
             P.quest_select(shape, cache, q, w.token_budget, page_ids, n_pages, ws_s)
@@ -305,16 +306,18 @@ def run_gpu(args, r: D.Rank):
         if c == 0:
             P.build_page_meta(shape, cache)
         elif c == 1:
-            P.route_pack(shape, d["v"], d["scores"], d["tok_class"], w.k_nominal, cache, total, status, ws_r)
+            P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)
         elif c == 2:
+            P.pack_values(shape, d["v"], cache, total, status, ws_r)
+        elif c == 3:
             if page_ids is not None:
                 P.quest_select(shape, cache, q, w.token_budget, page_ids, n_pages, ws_s)
         else:
             P.decode_attn(shape, cache, q, page_ids, n_pages, SM_SCALE, out, ws_a)
 
     per_call_ms = []
-    for c in range(4):
-        if c == 2 and page_ids is None:
+    for c in range(5):
+        if c == 3 and page_ids is None:
             per_call_ms.append(0.0)
             continue
         body = lambda c=c: [call_fn(c, j) for j in range(NQ)]
@@ -383,11 +386,11 @@ def run_gpu(args, r: D.Rank):
         gbs = ab[n] / (ms * 1e-3) / 1e9 if ms > 0 and ab[n] else 0.0
         per_kernel[n] = {"us": round(ms * 1e3, 2), "alg_bytes": ab[n], "GBps": round(gbs, 1),
                          "frac_of_" + peak_src: round(gbs / peak, 4), "frac_of_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
-    read_ms = per_call_ms[2] + per_call_ms[3]
+    read_ms = per_call_ms[3] + per_call_ms[4]
     read_bytes = ab["quest_select"] + ab["decode_attn"]
     read_gbs = read_bytes / (read_ms * 1e-3) / 1e9
-    # dominant call of the step (route_pack is a chain of five kernels, timed as one call)
-    single = {n: per_call_ms[c] for c, n in enumerate(names) if ab[n]}
+    # dominant single-kernel call of the step (route_mask is a chain of four kernels)
+    single = {n: per_call_ms[c] for c, n in enumerate(names) if ab[n] and n != "route_mask"}
     dom = max(single, key=single.get)
     roof = {"bound": "hbm", "kernel": KERNEL_OF[dom], "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
             "frac": round(per_kernel[dom]["GBps"] / peak, 4), "peak_source": peak_src + " copy bandwidth",
@@ -427,12 +430,15 @@ def run_gpu(args, r: D.Rank):
 
 
 KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kernel",
-             "decode_attn": "decode_attn_kernel",
-             "route_pack": "stc_route_pack call (route_hist_kernel x3 + route_mask_kernel + route_compact_kernel)"}
+             "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel"}
 
 # Per-launch DRAM traffic of the dominant kernel from the committed ncu capture
 # (profiles/), in bytes; None until a capture exists for that workload.
-TRAFFIC_NOTE: dict = {}
+TRAFFIC_NOTE: dict = {
+    # route_compact_kernel: 365.6 B of DRAM traffic per cached token (read 244.5 + write 121.1), from the ncu
+    # capture of a 4-sequence cfg4 case (profiles/), scaled by tokens to cfg1's 1,048,576 (problem, token) rows
+    ("cfg1", "pack_values"): 383.4e6,
+}
 
 
 # -------------------------------------------------------------------- reference arm

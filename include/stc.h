@@ -185,6 +185,22 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
                        int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes,
                        void* stream);
 
+/* stc_route_pack in its two halves, for callers that want the masks before the
+ * values are available (or want to time them apart).  stc_route_mask is the
+ * routing-mask rule of stc_route_pack (same passages, same arguments): it
+ * leaves in out->v_mask the groups every token keeps for certain and, in the
+ * workspace, the groups tied at the selection threshold and the per-tile
+ * counts.  stc_pack_values turns that into the final masks (ties resolved to
+ * the lowest flat indices), the offsets, the packed store, totals and status.
+ * It must be the next use of the same workspace after stc_route_mask, with
+ * the same shape, cache and mode.  The pair produces exactly the outputs of
+ * stc_route_pack.  ws: STC_OP_ROUTE_PACK for both. */
+int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_t* tok_class,
+                       int64_t class_head_stride, int32_t k_nominal, int32_t min_per_token, int32_t mode,
+                       const stc_cache* out, void* ws, size_t ws_bytes, void* stream);
+int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
+                        int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
 /* Routed decode attention (Section 3.3, attention equation): per query head h
  * with KV head h / (Hq/Hkv) and R = the valid tokens of the listed pages,
  *     s_t = sm_scale * q_h.k_t,  p = softmax over R of s,

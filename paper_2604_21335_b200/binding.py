@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values",
 )
 
 
@@ -75,6 +75,10 @@ def load_library():
         lib.stc_route_pack.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                        C.c_int32, C.c_int32, C.c_int32, C.POINTER(_Cache), C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.stc_route_mask.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32,
+                                       C.c_int32, C.POINTER(_Cache), C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.stc_pack_values.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_int32, C.POINTER(_Cache), C.c_void_p,
+                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_decode_attn.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
@@ -217,6 +221,27 @@ def route_pack(shape: Shape, v: torch.Tensor, scores: torch.Tensor, tok_class: O
         _ptr(tok_class, torch.uint8, "tok_class"), stride, k_nominal, min_per_token, mode, C.byref(cc),
         _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"),
         _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()), "stc_route_pack")
+
+
+def route_mask(shape: Shape, scores: torch.Tensor, tok_class: Optional[torch.Tensor], k_nominal: int,
+               cache: Cache, ws: torch.Tensor, min_per_token: int = 1, mode: int = MODE_GLOBAL) -> None:
+    """First half of route_pack: the routing masks (ties at the threshold are left in `ws`)."""
+    stride = shape.t_cap if (tok_class is not None and tok_class.dim() == 3) else 0
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_route_mask(
+        C.byref(cs), _ptr(scores, torch.float32, "scores"), _ptr(tok_class, torch.uint8, "tok_class"), stride,
+        k_nominal, min_per_token, mode, C.byref(cc), _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()),
+        "stc_route_mask")
+
+
+def pack_values(shape: Shape, v: torch.Tensor, cache: Cache, total_groups: torch.Tensor, status: torch.Tensor,
+                ws: torch.Tensor, mode: int = MODE_GLOBAL) -> None:
+    """Second half of route_pack: final masks, offsets and the packed value store."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_pack_values(
+        C.byref(cs), _ptr(v, torch.bfloat16, "v"), mode, C.byref(cc),
+        _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"),
+        _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()), "stc_pack_values")
 
 
 def decode_attn(shape: Shape, cache: Cache, q: torch.Tensor, page_ids: Optional[torch.Tensor],

@@ -77,7 +77,8 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
                               const uint8_t* tok_class, int64_t class_head_stride, int k_nominal,
                               int min_per_token, int mode, void* v_packed, uint16_t* v_mask,
                               uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups,
-                              int32_t* status, void* ws, cudaStream_t st);
+                              int32_t* status, void* ws, int phases /*1 = masks, 2 = pack, 3 = both*/,
+                              cudaStream_t st);
 
 struct AttnPlan { int n_workers, slots_cap; };   // warps that share the pages; partial slots per problem
 AttnPlan attn_plan(const Geom& g, int max_pages);

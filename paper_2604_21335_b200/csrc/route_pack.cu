@@ -451,9 +451,10 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
                               const uint8_t* tok_class, int64_t class_head_stride, int k_nominal,
                               int min_per_token, int mode, void* v_packed, uint16_t* v_mask,
                               uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups,
-                              int32_t* status, void* ws, cudaStream_t st) {
+                              int32_t* status, void* ws, int phases, cudaStream_t st) {
     if (g.problems == 0) return cudaSuccess;
     const RouteWs w = carve(g, ws);
+    const bool do_route = phases & 1, do_pack = phases & 2;
     const int n_tiles = (g.T + kTile - 1) / kTile;
     const long long n_cta = (long long)n_tiles * g.problems;
     if (n_cta > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
@@ -463,20 +464,22 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     const unsigned n_cta_scan = (unsigned)((n_tiles + tpc - 1) / tpc) * (unsigned)g.problems;
     const int64_t cls_h = class_head_stride;
     const int64_t cls_b = class_head_stride ? (int64_t)g.Hkv * class_head_stride : (int64_t)g.T;
-    cudaError_t e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
-    if (e != cudaSuccess) return e;
+    if (do_route) {
+        cudaError_t e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
+        if (e != cudaSuccess) return e;
+    }
 
 #define STC_ROUTE(S_)                                                                               \
     case S_: {                                                                                      \
-        if (mode == STC_MODE_GLOBAL)                                                                \
+        if (do_route && mode == STC_MODE_GLOBAL)                                                    \
             for (int pass = 0; pass < 3; ++pass)                                                    \
                 route_hist_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                             \
                     scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal, \
                     min_per_token, pass, w.state, w.hist);                                          \
-        route_mask_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                                     \
+        if (do_route) route_mask_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                                     \
             scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal,        \
             min_per_token, mode, w.state, v_mask, w.tie, w.tile_sums);                              \
-        route_compact_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                             \
+        if (do_pack) route_compact_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                             \
             static_cast<const uint4*>(v), g.seq_len, g.Hkv, g.T, n_tiles, mode, w.state,            \
             w.tile_sums, w.tie, v_mask, v_offs, static_cast<uint4*>(v_packed), cap_groups,          \
             total_groups, status);                                                                  \

@@ -103,11 +103,12 @@ int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const v
                                        static_cast<cudaStream_t>(stream)));
 }
 
-int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* scores,
-                       const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
-                       int32_t min_per_token, int32_t mode, const stc_cache* out,
-                       int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes,
-                       void* stream) {
+namespace {
+int32_t route_pack_phases(const stc_shape* shape, const void* v, const float* scores,
+                          const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
+                          int32_t min_per_token, int32_t mode, const stc_cache* out,
+                          int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, int phases,
+                          void* stream) {
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -116,15 +117,39 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
         return STC_ERR_INVALID_ARG;
     if (class_head_stride != 0 && class_head_stride != g.T) return STC_ERR_INVALID_ARG;
     if (empty(g)) return STC_OK;
-    if (!v || !scores || !out->v_packed || !out->v_mask || !out->v_offs || !total_groups || !status ||
-        out->cap_groups < 0)
+    if (!out->v_mask) return STC_ERR_INVALID_ARG;
+    if ((phases & 1) && !scores) return STC_ERR_INVALID_ARG;
+    if ((phases & 2) && (!v || !out->v_packed || !out->v_offs || !total_groups || !status || out->cap_groups < 0))
         return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, route_ws_bytes(g));
     if (rc != STC_OK) return rc;
     return cuda_rc(launch_route_pack(g, v, scores, tok_class, class_head_stride, k_nominal,
                                      min_per_token, mode, out->v_packed, out->v_mask, out->v_offs,
-                                     out->cap_groups, total_groups, status, ws,
+                                     out->cap_groups, total_groups, status, ws, phases,
                                      static_cast<cudaStream_t>(stream)));
+}
+}  // namespace
+
+int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* scores,
+                       const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
+                       int32_t min_per_token, int32_t mode, const stc_cache* out,
+                       int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes,
+                       void* stream) {
+    return route_pack_phases(shape, v, scores, tok_class, class_head_stride, k_nominal, min_per_token, mode,
+                             out, total_groups, status, ws, ws_bytes, 3, stream);
+}
+
+int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_t* tok_class,
+                       int64_t class_head_stride, int32_t k_nominal, int32_t min_per_token, int32_t mode,
+                       const stc_cache* out, void* ws, size_t ws_bytes, void* stream) {
+    return route_pack_phases(shape, nullptr, scores, tok_class, class_head_stride, k_nominal, min_per_token,
+                             mode, out, nullptr, nullptr, ws, ws_bytes, 1, stream);
+}
+
+int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
+                        int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+    return route_pack_phases(shape, v, nullptr, nullptr, 0, 0, 0, mode, out, total_groups, status, ws,
+                             ws_bytes, 2, stream);
 }
 
 int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const void* q,

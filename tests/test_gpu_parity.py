@@ -96,6 +96,27 @@ def test_routing_modes(kn, mpt, mode):
     full_parity(w, min_per_token=mpt, mode=mode)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+def test_route_mask_then_pack_values_equals_route_pack(mode):
+    w = W.shrink(W.get("cfg2"), batch=2, t_cache=2500, k_nominal=3)
+    d = W.make_inputs(w, DEV)
+    d["scores"] = torch.round(d["scores"] * 4) / 4            # ties at the threshold
+    g = H.gpu_pipeline(w, d, mode=mode)
+    shape = g["shape"]
+    c2 = P.Cache.allocate(shape, d["k"], g["cache"].cap_groups)
+    c2.v_packed.fill_(float("nan"))
+    total = torch.full_like(g["total"], -1); status = torch.full_like(g["status"], -1)
+    ws = Bd.new_workspace(shape, Bd.OP_ROUTE_PACK, device=DEV)
+    ws.fill_(0x5A)
+    P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, c2, ws, mode=mode)
+    P.pack_values(shape, d["v"], c2, total, status, ws, mode=mode)
+    torch.cuda.synchronize()
+    assert torch.equal(c2.v_mask, g["cache"].v_mask) and torch.equal(c2.v_offs, g["cache"].v_offs)
+    assert torch.equal(total, g["total"]) and torch.equal(status, g["status"])
+    n = int(total.max())
+    assert torch.equal(c2.v_packed[:, :, :n].view(torch.int16), g["cache"].v_packed[:, :, :n].view(torch.int16))
+
+
 def test_injected_ties_resolve_to_lower_indices():
     w = W.shrink(W.get("cfg0"), n_q_heads=2, n_kv_heads=2, t_cache=16 * 64, token_budget=16 * 10)
     d = W.make_inputs(w, DEV)
