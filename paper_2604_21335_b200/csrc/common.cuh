@@ -35,6 +35,15 @@ __device__ __forceinline__ uint4 ldg_nc16(const void* p) {
     return r;
 }
 
+// Same, asking L2 to fetch no more than the 64-byte granule around the address: for
+// gathers whose neighbours are mostly not wanted.
+__device__ __forceinline__ uint4 ldg_nc16_narrow(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::64B.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
 // Ampere-style asynchronous 16-byte copy global -> shared (L2 only), with
 // optional zero fill: src_bytes = 0 writes 16 zero bytes without reading.
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

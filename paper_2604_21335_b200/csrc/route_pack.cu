@@ -433,7 +433,7 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
                 const int64_t slot = (int64_t)s_offs[tl] + __popc(m & ((1u << grp) - 1u));
                 if (slot < cap_groups) {
                     where[u] = slot * OPG + (oct % OPG);
-                    val[u] = ldg_nc16(vrow + idx);
+                    val[u] = ldg_nc16_narrow(vrow + idx);
                 }
             }
         }
