@@ -77,6 +77,10 @@ CONFIGS: Dict[str, Workload] = {
     # LLaVA-1.5-7B-shaped cache: 128 text + 25% of 576 visual tokens
     "cfg3": Workload("cfg3", 32, 32, 32, _vlm_cache_len(128, 576, 0.25), 8, 3, None, "normal",
                      n_text=128, n_visual_total=576, visual_keep=0.25, seed=0x5C7C0003),
+    # cfg1 for all 32 layers of the model in one call: the layers' caches are stacked along the
+    # batch axis (the library treats every (batch, kv head) problem independently, so a stack
+    # of layers is just a larger batch) -- amortises the per-call latency of the small configs
+    "cfg1x32": Workload("cfg1x32", 32, 32, 32, 32768, 8, 4, 2048, "vnorm", seed=0x5C7C0011),
     # long-context GQA sweep base point (budget / k_nominal overridden per point)
     "cfg4": Workload("cfg4", 16, 32, 8, 131072, 8, 4, 4096, "normal", seed=0x5C7C0004),
 }
