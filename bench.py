@@ -435,9 +435,9 @@ KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kern
 # Per-launch DRAM traffic of the dominant kernel from the committed ncu capture
 # (profiles/), in bytes; None until a capture exists for that workload.
 TRAFFIC_NOTE: dict = {
-    # route_compact_kernel: 365.6 B of DRAM traffic per cached token (read 244.5 + write 121.1), from the ncu
-    # capture of a 4-sequence cfg4 case (profiles/), scaled by tokens to cfg1's 1,048,576 (problem, token) rows
-    ("cfg1", "pack_values"): 383.4e6,
+    # route_compact_kernel on this very workload: dram__bytes_read 205.7 MB + dram__bytes_write 83.0 MB per launch
+    # (profiles/traffic_bench_cfg1.md; part of the packed store is still in L2 when the kernel ends)
+    ("cfg1", "pack_values"): 288.7e6,
 }
 
 
