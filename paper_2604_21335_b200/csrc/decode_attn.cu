@@ -51,7 +51,7 @@ constexpr int kStagesDeep = 6;                   // one CTA per SM (calls too sm
 constexpr int kMaxGq = 8;
 constexpr int kCtasPerSm = 2;
 constexpr int kMinPagesPerWarp = 4;
-constexpr int kMaxSlots = 16;                    // partials per problem the merging warp handles (lane = slot, <= 32)
+constexpr int kMaxSlots = 32;                    // partials per problem the merging warp handles (lane = slot, <= 32)
 constexpr uint32_t kKeyBytes = kPage * kRowBytes;          // 4096
 constexpr uint32_t kStageBytes = 2 * kKeyBytes;            // keys + worst-case value span
 __host__ __device__ constexpr uint32_t ring_bytes(int stages) { return kWarps * stages * kStageBytes; }
@@ -222,7 +222,7 @@ decode_attn_kernel(const AttnArgs a) {
     int p_issue = (int)(x_lo / mp);              // its problem
     int slot_issue = (int)(x_lo - (long long)p_issue * mp);
 
-    auto issue = [&](int s) -> InFlight {        // bring position x_issue into stage s
+    auto issue = [&](int s, bool reuse) -> InFlight {   // bring position x_issue into stage s
         InFlight f{0, 0u, 0u};
         if (x_issue >= x_hi) return f;
         if (x_issue - win_base >= 32) { win_base = x_issue; fill_window(win_base); }
@@ -239,7 +239,7 @@ decode_attn_kernel(const AttnArgs a) {
             if (lane == 0) {
                 const uint32_t kb = (uint32_t)nv * kRowBytes, vb = groups * kGroupBytes;
                 const uint32_t bar = bars + 8 * s, dst = ring + (uint32_t)s * kStageBytes;
-                fence_proxy_async();             // the stage's earlier reads precede the new writes
+                if (reuse) fence_proxy_async();  // the stage's earlier reads precede the new writes
                 mbar_expect_tx(bar, kb + vb);
                 bulk_g2s(dst, a.k + row0 * kRowBytes, kb, bar);
                 if (vb)
@@ -558,7 +558,7 @@ decode_attn_kernel(const AttnArgs a) {
     // ---- main loop ----------------------------------------------------------------------------
     InFlight f[kStages];                          // f[0] = oldest page in flight, in stage s
 #pragma unroll
-    for (int i = 0; i < kStages; ++i) f[i] = issue(i);
+    for (int i = 0; i < kStages; ++i) f[i] = issue(i, false);
 
     int p_cur = (int)(x_lo / mp);
     int slot_cur = (int)(x_lo - (long long)p_cur * mp);
@@ -589,7 +589,7 @@ decode_attn_kernel(const AttnArgs a) {
         __syncwarp();
 #pragma unroll
         for (int i = 0; i + 1 < kStages; ++i) f[i] = f[i + 1];
-        f[kStages - 1] = issue(s);
+        f[kStages - 1] = issue(s, true);
         s = s + 1 == kStages ? 0 : s + 1;
         ++slot_cur;
         if (slot_cur == mp || n + 1 == count) {   // the range leaves this problem (one call site: finish is big)
