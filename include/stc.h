@@ -201,6 +201,26 @@ int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_
 int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
                         int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream);
 
+/* Streaming append (Section 3.4: "query-region tokens are not compressed" -- the
+ * tokens generated during decoding keep their full values).  For every sequence
+ * b the tokens old_len[b] <= t < len[b] (len = shape->seq_len AFTER the append,
+ * or t_cap when seq_len is NULL) have just been added: their keys are already in
+ * cache->k and their values in v (same [B][Hkv][T][128] layout as stc_route_pack;
+ * only the new rows are read).  The call
+ *   - stores all S groups of each new token behind the sequence's packed groups
+ *     (v_mask = all ones, v_offs advanced by S per token, v_offs[len] = total),
+ *   - recomputes kmin / kmax of every page that holds a new token, over all of
+ *     the page's valid tokens.
+ * The result equals stc_build_page_meta + stc_route_pack over the longer
+ * sequence with the new tokens in class FULL.  old_len: device i32 [B];
+ * max_new: upper bound of len[b] - old_len[b] (sizes the launch).
+ * total_groups / status as in stc_route_pack; a sequence whose lengths are
+ * inconsistent (old_len > len, or more than max_new new tokens) is left
+ * untouched with status STC_ERR_INVALID_ARG.  Needs no workspace. */
+int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const void* v,
+                          const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
+                          void* stream);
+
 /* Routed decode attention (Section 3.3, attention equation): per query head h
  * with KV head h / (Hq/Hkv) and R = the valid tokens of the listed pages,
  *     s_t = sm_scale * q_h.k_t,  p = softmax over R of s,

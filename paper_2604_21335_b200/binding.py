@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens",
 )
 
 
@@ -79,6 +79,8 @@ def load_library():
                                        C.c_int32, C.POINTER(_Cache), C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_pack_values.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_int32, C.POINTER(_Cache), C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.stc_append_tokens.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_decode_attn.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
@@ -242,6 +244,16 @@ def pack_values(shape: Shape, v: torch.Tensor, cache: Cache, total_groups: torch
         C.byref(cs), _ptr(v, torch.bfloat16, "v"), mode, C.byref(cc),
         _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"),
         _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()), "stc_pack_values")
+
+
+def append_tokens(shape: Shape, cache: Cache, v: torch.Tensor, old_len: torch.Tensor, max_new: int,
+                  total_groups: torch.Tensor, status: torch.Tensor) -> None:
+    """Tokens old_len[b] .. shape.seq_len[b] were just added: store their values in full, refresh page metadata."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_append_tokens(
+        C.byref(cs), C.byref(cc), _ptr(v, torch.bfloat16, "v"), _ptr(old_len, torch.int32, "old_len"), max_new,
+        _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"), _stream()),
+        "stc_append_tokens")
 
 
 def decode_attn(shape: Shape, cache: Cache, q: torch.Tensor, page_ids: Optional[torch.Tensor],

@@ -89,6 +89,11 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
                               int32_t* status, void* ws, int phases /*1 = masks, 2 = pack, 3 = both*/,
                               cudaStream_t st);
 
+cudaError_t launch_append(const Geom& g, const void* k, void* kmin, void* kmax, const void* v,
+                          const int32_t* old_len, int max_new, void* v_packed, uint16_t* v_mask,
+                          uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups, int32_t* status,
+                          cudaStream_t st);
+
 struct AttnPlan { int n_workers, slots_cap; };   // warps that share the pages; partial slots per problem
 AttnPlan attn_plan(const Geom& g, int max_pages);
 size_t attn_ws_bytes(const Geom& g, int max_pages);

@@ -152,6 +152,22 @@ int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, con
                              ws_bytes, 2, stream);
 }
 
+int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const void* v,
+                          const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
+                          void* stream) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (!cache || max_new < 0) return STC_ERR_INVALID_ARG;
+    if (empty(g) || max_new == 0) return STC_OK;
+    if (!cache->k || !cache->kmin || !cache->kmax || !cache->v_packed || !cache->v_mask || !cache->v_offs ||
+        cache->cap_groups < 0 || !v || !old_len || !total_groups || !status)
+        return STC_ERR_INVALID_ARG;
+    return cuda_rc(launch_append(g, cache->k, cache->kmin, cache->kmax, v, old_len, max_new, cache->v_packed,
+                                 cache->v_mask, cache->v_offs, cache->cap_groups, total_groups, status,
+                                 static_cast<cudaStream_t>(stream)));
+}
+
 int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const void* q,
                         const int32_t* page_ids, const int32_t* n_pages, int32_t max_pages,
                         float sm_scale, float* out, float* lse_opt, void* ws, size_t ws_bytes,
