@@ -245,3 +245,16 @@ def attend_batch(q, k, S, mask, page_ids, n_pages, scale, packed=None, offs=None
                              _p(ids), _p(npg), C.c_int32(0 if ids is None else ids.shape[2]),
                              C.c_double(scale), C.c_int32(use_dense), _p(out), _p(lse))
     return out, lse
+
+
+def router_logits(h, w, S, bias=None):
+    """h uint16 [B,T,d_model], w uint16 [Hkv*S,d_model], bias f32 [B,Hkv*S] or None -> f64 [B,Hkv,T,S]."""
+    B, T, dm = h.shape
+    N = w.shape[0]
+    Hkv = N // S
+    out = np.zeros((B, Hkv, T, S), np.float64)
+    b = None if bias is None else np.ascontiguousarray(bias, np.float32)
+    lib().stc_o_router_logits(C.c_int32(B), C.c_int32(Hkv), C.c_int32(T), C.c_int32(S), C.c_int32(dm),
+                              _p(np.ascontiguousarray(h), np.uint16), _p(np.ascontiguousarray(w), np.uint16),
+                              _p(b), _p(out))
+    return out

@@ -474,6 +474,34 @@ void stc_o_attend_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const
     }
 }
 
+/* ------------------------------------------------------------------------
+ * Value-group router (Appendix A.1 "Value-Group Router": a single linear
+ * projection from the layer input hidden state to S group logits; Section 3.4
+ * gives the LLM form a = g(h, s_Q), read here as the same linear map applied to
+ * [h ; s_Q], whose s_Q part is one additive vector per sequence).
+ *   h     [B][T][d_model]  bf16 hidden states
+ *   w     [Hkv*S][d_model] bf16 router weights, row hk*S + j = group j of KV head hk
+ *   bias  [B][Hkv*S] fp32 or NULL (the query-summary term)
+ *   out   [B][Hkv][T][S]   fp64 logits, the layout of the routing scores
+ * ---------------------------------------------------------------------- */
+void stc_o_router_logits(int32_t B, int32_t Hkv, int32_t T, int32_t S, int32_t d_model,
+                         const uint16_t* h, const uint16_t* w, const float* bias, double* out) {
+    int32_t N = Hkv * S;
+#pragma omp parallel for schedule(static)
+    for (int64_t bt = 0; bt < (int64_t)B * T; ++bt) {
+        int32_t b = (int32_t)(bt / T), t = (int32_t)(bt % T);
+        const uint16_t* hr = h + (size_t)bt * d_model;
+        for (int32_t n = 0; n < N; ++n) {
+            const uint16_t* wr = w + (size_t)n * d_model;
+            double acc = 0.0;
+            for (int32_t c = 0; c < d_model; ++c)
+                acc += (double)bf16_to_f32(hr[c]) * (double)bf16_to_f32(wr[c]);
+            if (bias) acc += (double)bias[(size_t)b * N + n];
+            out[(((size_t)b * Hkv + n / S) * T + t) * S + n % S] = acc;
+        }
+    }
+}
+
 int32_t stc_o_max_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

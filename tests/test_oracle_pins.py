@@ -380,6 +380,40 @@ def test_attend_page_subset_order_and_split_merge():
     assert m + math.log(wa + wb) == pytest.approx(lse, abs=1e-12)
 
 
+# ---------------------------------------------------------------------- router
+def test_router_logits_one_hot_rows_pick_hidden_channels_and_bias_adds():
+    g = rng(20)
+    B, T, dm, Hkv, S = 2, 5, 64, 2, 4
+    h = bf16(torch.randn(B, T, dm, generator=g))
+    w = np.zeros((Hkv * S, dm), np.uint16)
+    one = bf16(torch.tensor([1.0]))[0]
+    pick = [3, 17, 0, 63, 9, 9, 40, 5]                       # row n copies hidden channel pick[n]
+    for n, c in enumerate(pick):
+        w[n, c] = one
+    out = O.router_logits(h, w, S)
+    assert out.shape == (B, Hkv, T, S)
+    hf = f32(h).astype(np.float64)
+    for n, c in enumerate(pick):
+        np.testing.assert_array_equal(out[:, n // S, :, n % S], hf[:, :, c])
+    bias = np.arange(B * Hkv * S, dtype=np.float32).reshape(B, Hkv * S) / 4
+    out_b = O.router_logits(h, w, S, bias)
+    np.testing.assert_array_equal(out_b - out, bias.reshape(B, Hkv, 1, S).astype(np.float64) * np.ones((1, 1, T, 1)))
+
+
+def test_router_logits_hand_example_and_library_matmul():
+    # hand-worked: h = (1, 2, -3, 0.5), two rows of W
+    h = bf16(torch.tensor([[[1.0, 2.0, -3.0, 0.5]]]))
+    w = bf16(torch.tensor([[2.0, 0.0, 1.0, 4.0], [-1.0, 0.5, 0.0, 2.0]]))
+    out = O.router_logits(h, w, 2)
+    np.testing.assert_array_equal(out.ravel(), [2 - 3 + 2, -1 + 1 + 1])
+    # against the library matmul in fp64 (row n of W, token t -> out[b, n // S, t, n % S])
+    g = rng(21)
+    B, T, dm, Hkv, S = 2, 37, 96, 3, 8
+    hh, ww = bf16(torch.randn(B, T, dm, generator=g)), bf16(torch.randn(Hkv * S, dm, generator=g))
+    want = (f32(hh).astype(np.float64) @ f32(ww).astype(np.float64).T).reshape(B, T, Hkv, S).transpose(0, 2, 1, 3)
+    np.testing.assert_allclose(O.router_logits(hh, ww, S), want, rtol=0, atol=1e-12)
+
+
 # --------------------------------------------------------------- batched layer
 def test_batched_drivers_agree_with_single_problem_calls():
     from paper_2604_21335_b200 import workload as W
