@@ -201,6 +201,24 @@ int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_
 int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
                         int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream);
 
+/* Value-group router logits (Appendix A.1 "Value-Group Router": one linear
+ * projection from the layer's input hidden state to S group logits per KV
+ * head; Section 3.4's query-aware form g(h, s_Q) is the same projection with an
+ * additive per-sequence term, passed as bias_opt):
+ *     scores[b][hk][t][j] = sum_c h[b][t][c] * w[hk*S + j][c]  (+ bias_opt[b][hk*S + j])
+ *   h         bf16 [B][t_cap][d_model]      hidden states
+ *   w         bf16 [Hkv*S][d_model]         router weights
+ *   bias_opt  f32  [B][Hkv*S] or NULL
+ *   scores    f32  [B][Hkv][t_cap][S]       the layout stc_route_pack reads
+ * bf16 products, fp32 accumulation on the tensor cores (tcgen05 + TMA); all
+ * t_cap rows are computed.  Supported: d_model a multiple of 64; Hkv*S a
+ * multiple of 16 and either <= 256 or a multiple of 256 (else
+ * STC_ERR_UNSUPPORTED); h, w, bias, scores 16-byte aligned.  status_word:
+ * device i32 the call writes (STC_OK, or STC_ERR_TIMEOUT if a bounded wait on
+ * the device expired; scores are then unspecified).  Needs no workspace. */
+int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, const float* bias_opt,
+                          int32_t d_model, float* scores, int32_t* status_word, void* stream);
+
 /* Streaming append (Section 3.4: "query-region tokens are not compressed" -- the
  * tokens generated during decoding keep their full values).  For every sequence
  * b the tokens old_len[b] <= t < len[b] (len = shape->seq_len AFTER the append,

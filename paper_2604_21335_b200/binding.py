@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits",
 )
 
 
@@ -80,6 +80,8 @@ def load_library():
         lib.stc_pack_values.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_int32, C.POINTER(_Cache), C.c_void_p,
                                         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_append_tokens.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.stc_router_logits.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_decode_attn.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
@@ -254,6 +256,16 @@ def append_tokens(shape: Shape, cache: Cache, v: torch.Tensor, old_len: torch.Te
         C.byref(cs), C.byref(cc), _ptr(v, torch.bfloat16, "v"), _ptr(old_len, torch.int32, "old_len"), max_new,
         _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"), _stream()),
         "stc_append_tokens")
+
+
+def router_logits(shape: Shape, h: torch.Tensor, w: torch.Tensor, scores: torch.Tensor, status_word: torch.Tensor,
+                  bias: Optional[torch.Tensor] = None) -> None:
+    """scores[b,hk,t,j] = h[b,t,:] . w[hk*S+j,:] (+ bias[b,hk*S+j]); h bf16 [B,T,d_model], w bf16 [Hkv*S,d_model]."""
+    cs = shape.c()
+    _check(load_library().stc_router_logits(
+        C.byref(cs), _ptr(h, torch.bfloat16, "h"), _ptr(w, torch.bfloat16, "w"), _ptr(bias, torch.float32, "bias"),
+        h.shape[-1], _ptr(scores, torch.float32, "scores"), _ptr(status_word, torch.int32, "status_word"),
+        _stream()), "stc_router_logits")
 
 
 def decode_attn(shape: Shape, cache: Cache, q: torch.Tensor, page_ids: Optional[torch.Tensor],

@@ -152,6 +152,23 @@ int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, con
                              ws_bytes, 2, stream);
 }
 
+int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, const float* bias_opt,
+                          int32_t d_model, float* scores, int32_t* status_word, void* stream) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (d_model <= 0) return STC_ERR_INVALID_ARG;
+    const int n = g.Hkv * g.S;
+    if (d_model % 64 != 0 || n % 16 != 0 || (n > 256 && n % 256 != 0)) return STC_ERR_UNSUPPORTED;
+    if (empty(g)) return STC_OK;
+    if (!h || !w || !scores || !status_word) return STC_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(h) | reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(scores) |
+          reinterpret_cast<uintptr_t>(bias_opt)) & 15u) != 0)
+        return STC_ERR_INVALID_ARG;
+    return cuda_rc(launch_router_logits(g, h, w, bias_opt, d_model, scores, status_word,
+                                        static_cast<cudaStream_t>(stream)));
+}
+
 int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const void* v,
                           const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
                           void* stream) {
