@@ -6,7 +6,7 @@
 // GEMM with both operands K-major, bf16 in, fp32 accumulate.
 //
 // One CTA computes a 128-token x BN-logit tile (BN = all Hkv*S logits, <= 256):
-//   warp 0      one lane streams 64-wide K slices of both operands into a 4-stage
+//   warp 0      one lane streams 64-wide K slices of both operands into a 2..8-stage
 //               shared-memory ring with TMA (cp.async.bulk.tensor, 128-byte swizzle)
 //   warp 1      allocates the accumulator in tensor memory (128 lanes x BN columns);
 //               one lane issues tcgen05.mma (M128 x N(BN) x K16, four per slice) and
@@ -28,13 +28,13 @@ namespace {
 
 constexpr int kBM = 128;                 // tokens per CTA
 constexpr int kBK = 64;                  // K slice: 64 bf16 = one 128-byte swizzle row
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;            // ring depth = what fits in kRingBytes, at most this
 constexpr int kMaxBN = 256;
 constexpr int kThreads = 192;            // 6 warps: TMA, MMA, 4 x epilogue
 constexpr uint32_t kABytes = kBM * kBK * 2;              // 16 KiB
 constexpr uint32_t kBBytesMax = kMaxBN * kBK * 2;        // 32 KiB
-constexpr uint32_t kStageBytes = kABytes + kBBytesMax;   // 48 KiB, multiples of 1024 throughout
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers etc. */;
+constexpr uint32_t kRingBytes = 2 * (kABytes + kBBytesMax);  // 96 KiB: two CTAs per SM; 2 stages at BN = 256, 4 at BN = 64
+constexpr uint32_t kSmemBytes = kRingBytes + 1024 /* alignment slack */ + 256 /* barriers etc. */;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -106,17 +106,20 @@ struct RouterArgs {
     int BN;                 // logits per CTA tile (<= 256, multiple of 16)
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 router_logits_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
                      const RouterArgs a) {
     extern __shared__ unsigned char smem_raw[];
     // 128-byte-swizzled tiles need 1024-byte aligned bases
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t ctrl = base + kStages * kStageBytes;          // barriers, TMEM address, abort flag
-    const uint32_t full0 = ctrl, empty0 = ctrl + 8 * kStages, tmem_full = ctrl + 16 * kStages;
+    const uint32_t ctrl = base + kRingBytes;                     // barriers, TMEM address, abort flag
+    const uint32_t full0 = ctrl, empty0 = ctrl + 8 * kMaxStages, tmem_full = ctrl + 16 * kMaxStages;
     unsigned char* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + 16 * kStages + 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 16 * kStages + 12);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + 16 * kMaxStages + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + 16 * kMaxStages + 12);
+    // a stage = the 128 x 64 slice of h and the BN x 64 slice of w (both multiples of 1024 bytes)
+    const uint32_t kStageBytes = kABytes + (uint32_t)a.BN * kBK * 2;
+    const int kStages = min(kMaxStages, (int)(kRingBytes / kStageBytes));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * kBM, n0 = blockIdx.y * a.BN;
@@ -134,7 +137,7 @@ router_logits_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
     }
     if (warp == 1) {                                  // whole warp: allocate the accumulator
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(ctrl + 16 * kStages + 8), "r"(tmem_cols) : "memory");
+                     ::"r"(ctrl + 16 * kMaxStages + 8), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
