@@ -441,6 +441,57 @@ TRAFFIC_NOTE: dict = {
 }
 
 
+# ------------------------------------------------------------------ router (a "next" row)
+D_MODEL = {"cfg2": 3584}                                    # Qwen2.5-7B; the other shapes are 4096-wide models
+
+
+def run_router(args):
+    """Times stc_router_logits alone on the workload's shape (not part of the step) and prints one line."""
+    import paper_2604_21335_b200 as P
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = select_workload(args)
+    B, T, Hkv, S = w.batch, w.t_cache, w.n_kv_heads, w.n_groups
+    dm = D_MODEL.get(args.workload, 4096)
+    g = torch.Generator(device=dev); g.manual_seed(w.seed ^ 0x707)
+    NH = 2 if B * T * dm * 2 > (8 << 30) else 4                # rotating hidden-state sets, all larger than L2
+    hs = [torch.randn(B, T, dm, generator=g, device=dev).to(torch.bfloat16) for _ in range(NH)]
+    wt = (torch.randn(Hkv * S, dm, generator=g, device=dev) / dm ** 0.5).to(torch.bfloat16)
+    sc = torch.empty(B, Hkv, T, S, dtype=torch.float32, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    shape = P.Shape(B, Hkv, Hkv, S, T)
+    for i in range(max(args.warmup, 3)):
+        P.router_logits(shape, hs[i % NH], wt, sc, st)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    K = args.steps
+    e0.record()
+    for i in range(K):
+        P.router_logits(shape, hs[i % NH], wt, sc, st)
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(st[0]) == 0
+    us = e0.elapsed_time(e1) * 1e3 / K
+    M, N = B * T, Hkv * S
+    flops, nbytes = 2.0 * M * N * dm, M * dm * 2 + N * dm * 2 + M * N * 4
+    peak_gbs, src = peaks()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak_tf = float(json.load(f)["bf16_tflops"])
+    except Exception:
+        peak_tf = 1590.0
+    tf, gbs = flops / us / 1e6, nbytes / us / 1e3
+    bound = "hbm" if nbytes / peak_gbs > flops / (peak_tf * 1e3) else "tensor"
+    print(json.dumps({
+        "metric": "router_logits", "us": round(us, 2), "TFLOPs": round(tf, 1), "GBps": round(gbs, 1),
+        "config": {"workload": f"{w.name}: tokens {M}, logits {N}, d_model {dm}"},
+        "roofline": {"bound": bound, "achieved": round(gbs if bound == "hbm" else tf, 1),
+                     "peak": peak_gbs if bound == "hbm" else peak_tf, "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                     "frac": round((gbs / peak_gbs) if bound == "hbm" else (tf / peak_tf), 4),
+                     "peak_source": src, "traffic": None},
+        "steps": K, "data": "synthetic", "dtype": "bf16"}), flush=True)
+
+
 # -------------------------------------------------------------------- reference arm
 def run_reference(args, r: D.Rank):
     if not r.is_main:
@@ -502,6 +553,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--only", default=None, choices=["router"], help="time one extra kernel instead of the step")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
@@ -513,6 +565,11 @@ def main():
         if world > 1 and rank != 0:
             return                                           # rank 0 alone runs the CPU arm
         run_reference(args, D.Rank())
+        return
+    if args.only == "router":
+        args.steps = 20 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else args.warmup
+        run_router(args)
         return
     args.steps = 300 if args.steps is None else args.steps
     args.warmup = 5 if args.warmup is None else args.warmup
