@@ -221,19 +221,30 @@ def run_gpu(args, r: D.Rank):
     names = ["page_meta", "route_mask", "pack_values", "quest_select", "decode_attn"]
     launches_per_step = 1 + 5 + (1 if page_ids is not None else 0) + 1   # route_mask = 3 histogram passes + mask
 
-    def step(i, ev=None):
-        q = qs[i % NQ]
-        if ev: ev[0].record()
-        P.build_page_meta(shape, cache)
-        if ev: ev[1].record()
+    # The key side (page metadata, page selection) and the value side (routing, packing) of a
+    # pass touch disjoint data, so they run on two streams and join before the attention call;
+    # --serial puts all five calls on one stream.
+    side = None if args.serial else torch.cuda.Stream(device=dev)
+
+    def value_side():
         P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)     # stc_route_pack, first half
         P.pack_values(shape, d["v"], cache, total, status, ws_r)                       # ... second half
-        if ev: ev[2].record()
+
+    def step(i):
+        q = qs[i % NQ]
+        main = torch.cuda.current_stream()
+        if side is not None:
+            side.wait_stream(main)
+            with torch.cuda.stream(side):
+                value_side()
+        P.build_page_meta(shape, cache)
+        if side is None:
+            value_side()
         if page_ids is not None:
             P.quest_select(shape, cache, q, w.token_budget, page_ids, n_pages, ws_s)
-        if ev: ev[3].record()
+        if side is not None:
+            main.wait_stream(side)
         P.decode_attn(shape, cache, q, page_ids, n_pages, SM_SCALE, out, ws_a)
-        if ev: ev[4].record()
 
     W_ = max(args.warmup, 3)
     for i in range(W_):
@@ -404,7 +415,8 @@ def run_gpu(args, r: D.Rank):
                                "(page_meta + route_pack + quest_select + decode_attn)",
                    "l2": "inputs larger than L2 (K+V %.0f MiB re-read every step), %d rotating query sets"
                          % ((d["k"].numel() + d["v"].numel()) * 2 / 2 ** 20, NQ),
-                   "replicas": "one independent batch per rank, no collective"},
+                   "replicas": "one independent batch per rank, no collective",
+                   "streams": "one" if args.serial else "two (key side | value side, joined before decode_attn)"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "launch": launch_mode,
         "roofline": roof,
         "per_call": per_kernel,
@@ -553,6 +565,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--serial", action="store_true", help="all calls of a step on one stream")
     ap.add_argument("--only", default=None, choices=["router"], help="time one extra kernel instead of the step")
     args = ap.parse_args()
     if args.impl == "reference":
