@@ -219,7 +219,7 @@ def run_gpu(args, r: D.Rank):
     ws_a = Bd.new_workspace(shape, Bd.OP_DECODE_ATTN, max_pages, device=dev)
     qs = [d["q"][i].contiguous() for i in range(NQ)]
     names = ["page_meta", "route_mask", "pack_values", "quest_select", "decode_attn"]
-    launches_per_step = 1 + 5 + (1 if page_ids is not None else 0) + 1   # route_mask = 3 histogram passes + mask
+    launches_per_step = 1 + 2 + (1 if page_ids is not None else 0) + 1   # route_pack = select kernel + compact kernel
 
     # The key side (page metadata, page selection) and the value side (routing, packing) of a
     # pass touch disjoint data, so they run on two streams and join before the attention call;
@@ -442,7 +442,8 @@ def run_gpu(args, r: D.Rank):
 
 
 KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kernel",
-             "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel"}
+             "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel",
+             "route_mask": "route_select_kernel"}
 
 # Per-launch DRAM traffic of the dominant kernel from the committed ncu capture
 # (profiles/), in bytes; None until a capture exists for that workload.

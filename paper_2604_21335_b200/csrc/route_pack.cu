@@ -6,21 +6,23 @@
 // the lower flat index.  `take` depends on the routed-token count, which only
 // the device knows, so everything is resolved on the device:
 //
+//   select kernel (one persistent cooperative launch):
 //   hist pass 0/1/2  radix select (11+11+10 bits) of the take-th largest key
-//                    among the candidates; each CTA histograms a 1024-token
-//                    tile in shared memory and merges into the problem's
+//                    among the candidates; each CTA histograms its units of a
+//                    problem in shared memory and merges into the problem's
 //                    global histogram; the CTA that arrives last (atomic
-//                    ticket, nobody waits) picks the digit for the next pass.
-//   mask             per token: definite bits (reserved, FULL, key > tau) and
-//                    tie bits (key == tau); per-tile counts of both.
-//   compact          per tile: exclusive scan of the counts (tile base from the
-//                    preceding tiles' sums), ties kept in flat-index order
+//                    ticket) picks the digit and publishes it; CTAs wait (with
+//                    a time limit) for the digits of the problems they scan.
+//   mask pass        per token: definite bits (reserved, FULL, key > tau) and
+//                    tie bits (key == tau); per-unit counts of both.
+//   compact kernel   per tile: exclusive scan of the counts (tile base from the
+//                    preceding units' sums), ties kept in flat-index order
 //                    until the remaining rank is used up, final mask + offsets
 //                    written, kept 16-byte chunks of V copied to the store.
 //
 // PER_TOKEN mode skips the histogram passes (the mask is local to a token).
-// HBM traffic: scores 4x (3 passes + mask; 1x in PER_TOKEN mode), kept part of
-// V once in and once out.
+// HBM traffic: scores 4x (3 passes + mask, from L2 when they fit; 1x in PER_TOKEN
+// mode), kept part of V once in and once out.
 #include "common.cuh"
 
 namespace stc {
@@ -28,18 +30,22 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kTile = 1024;                   // tokens per CTA in every kernel here
+constexpr int kTile = 1024;                   // tokens per CTA of the compaction kernel
+constexpr int kUnit = kThreads;               // tokens per unit of the score scans (one per thread)
+constexpr int kUnitsPerTile = kTile / kUnit;
 constexpr int kTokPerThread = kTile / kThreads;
 constexpr int kBins = 2048;
 
 // state words per problem
-enum { ST_NROUTED = 0, ST_PREFIX, ST_KREM, ST_FLAGS, ST_TICKET0, ST_TICKET1, ST_TICKET2, ST_PAD, ST_WORDS };
+enum { ST_NROUTED = 0, ST_PREFIX, ST_KREM, ST_FLAGS, ST_TICKET0, ST_TICKET1, ST_TICKET2, ST_DONE, ST_WORDS };
 enum { FL_NONE = 1, FL_BUDGET = 2 };          // nothing beyond the reserved groups / budget error
+// ST_DONE = histogram passes resolved so far (3 = threshold final)
 
 struct RouteWs {
     uint32_t* state;      // [problems][ST_WORDS]
     uint32_t* hist;       // [problems][3][kBins]
-    uint32_t* tile_sums;  // [problems][n_tiles][2]
+    uint32_t* abort_word; // set when a bounded wait gave up
+    uint32_t* unit_sums;  // [problems][units]: definite count | tie count << 16
     uint16_t* tie;        // [problems][T]
     size_t zero_bytes;    // leading bytes (state + hist) cleared per call
     size_t total_bytes;
@@ -50,21 +56,19 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 RouteWs carve(const Geom& g, void* ws) {
     RouteWs r;
     char* p = static_cast<char*>(ws);
-    const int n_tiles = (g.T + kTile - 1) / kTile;
+    const int n_units = (g.T + kUnit - 1) / kUnit;
     size_t o = 0;
     r.state = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * ST_WORDS * 4);
     r.hist = reinterpret_cast<uint32_t*>(p + o);  o += align256((size_t)g.problems * 3 * kBins * 4);
+    r.abort_word = reinterpret_cast<uint32_t*>(p + o); o += 256;
     r.zero_bytes = o;
-    r.tile_sums = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * n_tiles * 2 * 4);
+    r.unit_sums = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * n_units * 4);
     r.tie = reinterpret_cast<uint16_t*>(p + o);   o += align256((size_t)g.problems * g.T * 2);
     r.total_bytes = o;
     return r;
 }
 
 __device__ __forceinline__ int pass_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
-__device__ __forceinline__ uint32_t pass_digit(uint32_t key, int pass) {
-    return pass == 2 ? (key & 1023u) : ((key >> pass_shift(pass)) & 2047u);
-}
 __device__ __forceinline__ uint32_t pass_himask(int pass) {
     return pass == 0 ? 0u : (pass == 1 ? 0xFFE00000u : 0xFFFFFC00u);
 }
@@ -99,10 +103,9 @@ __device__ __forceinline__ void load_raw(const float* __restrict__ row, uint4 (&
 #pragma unroll
     for (int i = 0; i < S / 4; ++i) raw[i] = __ldg(p + i);   // L1-allocating: the row's 16-byte pieces share sectors
 }
-// Scores of one token -> order-preserving keys; best = first maximum (tracked by
-// value, so no register array is indexed at run time).
+// Scores of one token -> order-preserving keys.
 template <int S>
-__device__ __forceinline__ void make_keys(const uint4 (&raw)[S / 4], uint32_t (&key)[S], int& best) {
+__device__ __forceinline__ void make_keys(const uint4 (&raw)[S / 4], uint32_t (&key)[S]) {
 #pragma unroll
     for (int i = 0; i < S / 4; ++i) {
         const uint4 w = raw[i];
@@ -111,14 +114,19 @@ __device__ __forceinline__ void make_keys(const uint4 (&raw)[S / 4], uint32_t (&
         key[4 * i + 2] = float_key(__uint_as_float(w.z));
         key[4 * i + 3] = float_key(__uint_as_float(w.w));
     }
+}
+// Index of the first maximum (tracked by value, so no register array is indexed at run time).
+template <int S>
+__device__ __forceinline__ int first_max(const uint32_t (&key)[S]) {
     uint32_t bk = key[0];
-    best = 0;
+    int best = 0;
 #pragma unroll
     for (int j = 1; j < S; ++j) {
         const bool up = key[j] > bk;
         bk = up ? key[j] : bk;
         best = up ? j : best;
     }
+    return best;
 }
 
 __device__ __forceinline__ int token_class(const uint8_t* cls, int t, int len) {
@@ -153,193 +161,262 @@ __device__ void pick_digit(const uint32_t* __restrict__ hist, int nbins, uint32_
     __syncthreads();
 }
 
-template <int S>
-__global__ void __launch_bounds__(kThreads)
-route_hist_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
-                  int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int n_tiles,
-                  int tiles_per_cta, int k_nominal, int min_per_token, int pass,
-                  uint32_t* __restrict__ state_all, uint32_t* __restrict__ hist_all) {
-    __shared__ uint32_t shist[kBins];
-    __shared__ uint32_t s_w[kWarps];
-    __shared__ uint32_t s_pick[2];
-    __shared__ int s_last;
+// ---- bounded cross-CTA hand-off -------------------------------------------------
+constexpr uint64_t kWaitNs = 2000000000ull;   // a wait that lasts this long gives up and reports a time-out
 
-    const int n_groups = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
-    const int problem = blockIdx.x / n_groups, group = blockIdx.x - problem * n_groups;
-    const int b = problem / Hkv, hk = problem - b * Hkv;
-    const int len = clamp_len(seq_len, b, T);
-    uint32_t* state = state_all + (size_t)problem * ST_WORDS;
-    uint32_t* hist = hist_all + ((size_t)problem * 3 + pass) * kBins;
-    const int tid = threadIdx.x;
-
-    uint32_t prefix = 0;
-    if (pass > 0) {
-        if (__ldcg(state + ST_FLAGS) != 0u) return;      // nothing to select / budget error
-        prefix = __ldcg(state + ST_PREFIX);
-    }
-    const uint32_t himask = pass_himask(pass);
-    const int dshift = pass_shift(pass);
-    const uint32_t dmask = pass == 2 ? 1023u : 2047u;
-    for (int i = tid; i < kBins; i += kThreads) shist[i] = 0;
-    __syncthreads();
-
-    const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
-    uint32_t n_routed = 0;
-    // several 1024-token tiles per CTA: the shared histogram is cleared and flushed once
-    const int tile_end = min(n_tiles, (group + 1) * tiles_per_cta);
-#pragma unroll 1
-    for (int tile = group * tiles_per_cta; tile < tile_end; ++tile) {
-        if (tile * kTile >= len) break;
-        uint4 raw[kTokPerThread][S / 4];          // all of the thread's loads are in flight before the first use
-        bool routed[kTokPerThread];
-#pragma unroll
-        for (int i = 0; i < kTokPerThread; ++i) {
-            const int t = tile * kTile + i * kThreads + tid;
-            routed[i] = token_class(c, t, len) == STC_CLS_ROUTED;
-            if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
-        }
-#pragma unroll
-        for (int i = 0; i < kTokPerThread; ++i) {
-            if (!routed[i]) continue;
-            ++n_routed;
-            uint32_t key[S];
-            int best;
-            make_keys<S>(raw[i], key, best);
-#pragma unroll
-            const int skip = min_per_token ? best : -1;
-#pragma unroll
-            for (int j = 0; j < S; ++j)
-                if (j != skip && (key[j] & himask) == prefix) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
-        }
-    }
-    __syncthreads();
-    for (int i = tid; i < kBins; i += kThreads) {
-        uint32_t v = shist[i];
-        if (v) atomicAdd(hist + i, v);
-    }
-    if (pass == 0) {
-        uint32_t tot;
-        block_excl_scan(n_routed, s_w, &tot);
-        if (tid == 0 && tot) atomicAdd(state + ST_NROUTED, tot);
-    }
-
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(state + ST_TICKET0 + pass, 1u) == (unsigned)(n_groups - 1));
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-
-    uint32_t krem;
-    if (pass == 0) {
-        const uint64_t n = __ldcg(state + ST_NROUTED);
-        const uint64_t m_total = n * (uint64_t)k_nominal;
-        uint32_t flags = 0;
-        if (min_per_token && m_total < n) flags = FL_BUDGET;
-        const uint64_t take = m_total - (min_per_token ? n : 0);
-        if (!flags && take == 0) flags = FL_NONE;
-        if (flags) {
-            if (tid == 0) { state[ST_FLAGS] = flags; state[ST_PREFIX] = 0; state[ST_KREM] = 0; }
-            return;
-        }
-        krem = (uint32_t)take;
-    } else {
-        krem = __ldcg(state + ST_KREM);
-    }
-    pick_digit(hist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
-    if (tid == 0) {
-        state[ST_PREFIX] = prefix | (s_pick[0] << pass_shift(pass));
-        state[ST_KREM] = s_pick[1];
-    }
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-template <int S>
-__global__ void __launch_bounds__(kThreads)
-route_mask_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
-                  int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int n_tiles,
-                  int tiles_per_cta, int k_nominal, int min_per_token, int mode,
-                  const uint32_t* __restrict__ state_all, uint16_t* __restrict__ v_mask,
-                  uint16_t* __restrict__ tie_all, uint32_t* __restrict__ tile_sums) {
-    __shared__ uint32_t s_w[kWarps];
-    const int n_groups = (n_tiles + tiles_per_cta - 1) / tiles_per_cta;
-    const int problem = blockIdx.x / n_groups, group = blockIdx.x - problem * n_groups;
-    const int b = problem / Hkv, hk = problem - b * Hkv;
-    const int len = clamp_len(seq_len, b, T);
-    const int tid = threadIdx.x;
-    const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
-
-    uint32_t tau = 0, flags = 0;
-    if (mode == STC_MODE_GLOBAL) {
-        const uint32_t* state = state_all + (size_t)problem * ST_WORDS;
-        flags = __ldcg(state + ST_FLAGS);
-        tau = __ldcg(state + ST_PREFIX);
-    }
-    const int tile_end = min(n_tiles, (group + 1) * tiles_per_cta);
-#pragma unroll 1
-    for (int tile = group * tiles_per_cta; tile < tile_end; ++tile) {
-    uint32_t n_def = 0, n_tie = 0;
-    uint4 raw[kTokPerThread][S / 4];              // loads first, arithmetic after
-    int cls_of[kTokPerThread];
-#pragma unroll
-    for (int i = 0; i < kTokPerThread; ++i) {
-        const int t = tile * kTile + i * kThreads + tid;
-        cls_of[i] = t < T ? token_class(c, t, len) : STC_CLS_DROP;
-        if (cls_of[i] == STC_CLS_ROUTED && !(flags & FL_BUDGET))
-            load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
-    }
-#pragma unroll
-    for (int i = 0; i < kTokPerThread; ++i) {
-        const int t = tile * kTile + i * kThreads + tid;
-        if (t >= T) continue;
-        const int cl = cls_of[i];
-        uint32_t def = 0, tie = 0;
-        if (flags & FL_BUDGET) {
-            def = 0;
-        } else if (cl == STC_CLS_FULL) {
-            def = (1u << S) - 1u;
-        } else if (cl == STC_CLS_ROUTED) {
-            uint32_t key[S];
-            int best;
-            make_keys<S>(raw[i], key, best);
-            if (mode == STC_MODE_PER_TOKEN) {
-#pragma unroll
-                for (int j = 0; j < S; ++j) {
-                    int rank = 0;
-#pragma unroll
-                    for (int i2 = 0; i2 < S; ++i2)
-                        rank += (key[i2] > key[j]) || (key[i2] == key[j] && i2 < j);
-                    if (rank < k_nominal) def |= 1u << j;
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < S; ++j) {
-                    if (min_per_token && j == best) { def |= 1u << j; continue; }
-                    if (flags & FL_NONE) continue;
-                    if (key[j] > tau) def |= 1u << j;
-                    else if (key[j] == tau) tie |= 1u << j;
-                }
+// Wait until `need` passes of the problem are resolved, then broadcast its state:
+// s_bc = {ok, flags, prefix, krem}.  False (for the whole CTA) after a time-out or when
+// another CTA has already given up.
+__device__ __forceinline__ bool wait_done(const uint32_t* state, uint32_t need, uint32_t* s_bc,
+                                          uint32_t* abort_word) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t ok = 1;
+        if (ld_acquire(state + ST_DONE) < need) {
+            const uint64_t t0 = globaltimer_ns();
+            while (ld_acquire(state + ST_DONE) < need) {
+                __nanosleep(100);
+                if (globaltimer_ns() - t0 > kWaitNs || ld_acquire(abort_word) != 0u) { ok = 0; break; }
             }
         }
-        v_mask[(size_t)problem * T + t] = (uint16_t)def;
-        tie_all[(size_t)problem * T + t] = (uint16_t)tie;
-        n_def += __popc(def);
-        n_tie += __popc(tie);
+        if (!ok) atomicExch(abort_word, 1u);
+        s_bc[0] = ok;
+        s_bc[1] = __ldcg(state + ST_FLAGS);
+        s_bc[2] = __ldcg(state + ST_PREFIX);
+        s_bc[3] = __ldcg(state + ST_KREM);
     }
-    uint32_t tot_def, tot_tie;
-    block_excl_scan(n_def, s_w, &tot_def);
-    block_excl_scan(n_tie, s_w, &tot_tie);
-    if (tid == 0) {
-        tile_sums[((size_t)problem * n_tiles + tile) * 2 + 0] = tot_def;
-        tile_sums[((size_t)problem * n_tiles + tile) * 2 + 1] = tot_tie;
+    __syncthreads();
+    return s_bc[0] != 0u;
+}
+
+// One persistent, cooperatively launched kernel (every CTA is resident, so a CTA may
+// wait for a digit another CTA publishes): the three histogram passes and the mask
+// pass.  Work is cut into units of 256 tokens (one per thread); a CTA owns a fixed,
+// contiguous range of the flat (problem, unit) sequence in every pass, and works through
+// it one segment (its units of one problem) at a time.
+template <int S>
+__global__ void __launch_bounds__(kThreads, 4)
+route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
+                    int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int upp,
+                    int k_nominal, int min_per_token, int mode, uint32_t* __restrict__ state_all,
+                    uint32_t* __restrict__ hist_all, uint32_t* __restrict__ abort_word,
+                    uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
+                    uint32_t* __restrict__ unit_sums, long long total_units) {
+    constexpr int kBatch = 32 / S;               // tokens in flight per thread (32 score registers)
+    __shared__ uint32_t shist[kBins];
+    __shared__ uint32_t s_w[kWarps];
+    __shared__ uint32_t s_red[kBatch][kWarps];
+    __shared__ uint32_t s_pick[2];
+    __shared__ uint32_t s_bc[4];
+    __shared__ int s_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long x0 = total_units * blockIdx.x / gridDim.x;
+    const long long x1 = total_units * (blockIdx.x + 1) / gridDim.x;
+    const int n_pass = mode == STC_MODE_GLOBAL ? 3 : 0;
+
+#pragma unroll 1
+    for (int pass = 0; pass < n_pass; ++pass) {
+        const uint32_t himask = pass_himask(pass);
+        const int dshift = pass_shift(pass);
+        const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+#pragma unroll 1
+        for (long long x = x0; x < x1;) {
+            const int problem = (int)(x / upp);
+            const int u0 = (int)(x - (long long)problem * upp);
+            const int n = (int)min((long long)(upp - u0), x1 - x);
+            x += n;
+            const int b = problem / Hkv, hk = problem - b * Hkv;
+            const int len = clamp_len(seq_len, b, T);
+            uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+            uint32_t* hist = hist_all + ((size_t)problem * 3 + pass) * kBins;
+            uint32_t prefix = 0, krem_in = 0;
+            if (pass > 0) {
+                if (!wait_done(state, (uint32_t)pass, s_bc, abort_word)) return;
+                if (s_bc[1] != 0u) continue;             // nothing to select / budget error: resolved in pass 0
+                prefix = s_bc[2];
+                krem_in = s_bc[3];
+            }
+            for (int i = tid; i < kBins; i += kThreads) shist[i] = 0;
+            __syncthreads();
+
+            const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+            uint32_t n_routed = 0;
+#pragma unroll 1
+            for (int u = u0; u < u0 + n; u += kBatch) {
+                if (u * kUnit >= len) break;
+                uint4 raw[kBatch][S / 4];                // all of the thread's loads are in flight before the first use
+                bool routed[kBatch];
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) {
+                    const int t = (u + i) * kUnit + tid;
+                    routed[i] = u + i < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
+                    if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) {
+                    if (!routed[i]) continue;
+                    ++n_routed;
+                    uint32_t key[S];
+                    make_keys<S>(raw[i], key);
+                    uint32_t cand = 0;                   // keys still in the running for this pass
+#pragma unroll
+                    for (int j = 0; j < S; ++j) cand |= ((key[j] & himask) == prefix ? 1u : 0u) << j;
+                    if (cand == 0u) continue;
+                    if (min_per_token) cand &= ~(1u << first_max<S>(key));
+#pragma unroll
+                    for (int j = 0; j < S; ++j)
+                        if ((cand >> j) & 1u) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
+                }
+            }
+            __syncthreads();
+            for (int i = tid; i < kBins; i += kThreads) {
+                const uint32_t v = shist[i];
+                if (v) atomicAdd(hist + i, v);
+            }
+            if (pass == 0) {
+                uint32_t tot;
+                block_excl_scan(n_routed, s_w, &tot);
+                if (tid == 0 && tot) atomicAdd(state + ST_NROUTED, tot);
+            }
+            __threadfence();
+            __syncthreads();
+            if (tid == 0)
+                s_last = (atomicAdd(state + ST_TICKET0 + pass, (unsigned)n) + (unsigned)n == (unsigned)upp);
+            __syncthreads();
+            if (!s_last) continue;
+            __threadfence();
+
+            // the CTA that completed the problem's pass picks the digit and publishes it
+            uint32_t krem = krem_in, flags = 0;
+            if (pass == 0) {
+                const uint64_t nr = __ldcg(state + ST_NROUTED);
+                const uint64_t m_total = nr * (uint64_t)k_nominal;
+                if (min_per_token && m_total < nr) flags = FL_BUDGET;
+                const uint64_t take = m_total - (min_per_token ? nr : 0);
+                if (!flags && take == 0) flags = FL_NONE;
+                krem = (uint32_t)take;
+            }
+            if (flags) {
+                if (tid == 0) { state[ST_FLAGS] = flags; state[ST_PREFIX] = 0; state[ST_KREM] = 0; }
+            } else {
+                pick_digit(hist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
+                if (tid == 0) {
+                    state[ST_PREFIX] = prefix | (s_pick[0] << pass_shift(pass));
+                    state[ST_KREM] = s_pick[1];
+                }
+            }
+            if (tid == 0) {
+                __threadfence();
+                st_release(state + ST_DONE, flags ? 3u : (uint32_t)(pass + 1));
+            }
+        }
     }
+
+    // ---- mask pass: definite bits, tie bits and their per-unit counts ------------------
+#pragma unroll 1
+    for (long long x = x0; x < x1;) {
+        const int problem = (int)(x / upp);
+        const int u0 = (int)(x - (long long)problem * upp);
+        const int n = (int)min((long long)(upp - u0), x1 - x);
+        x += n;
+        const int b = problem / Hkv, hk = problem - b * Hkv;
+        const int len = clamp_len(seq_len, b, T);
+        const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+        uint32_t tau = 0, flags = 0;
+        if (mode == STC_MODE_GLOBAL) {
+            if (!wait_done(state_all + (size_t)problem * ST_WORDS, 3u, s_bc, abort_word)) return;
+            flags = s_bc[1];
+            tau = s_bc[2];
+        }
+#pragma unroll 1
+        for (int u = u0; u < u0 + n; u += kBatch) {
+            uint4 raw[kBatch][S / 4];
+            int cls_of[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int t = (u + i) * kUnit + tid;
+                cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
+                if (cls_of[i] == STC_CLS_ROUTED && !(flags & FL_BUDGET))
+                    load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int t = (u + i) * kUnit + tid;
+                const int cl = cls_of[i];
+                uint32_t def = 0, tie = 0;
+                if (flags & FL_BUDGET) {
+                    def = 0;
+                } else if (cl == STC_CLS_FULL) {
+                    def = (1u << S) - 1u;
+                } else if (cl == STC_CLS_ROUTED) {
+                    uint32_t key[S];
+                    make_keys<S>(raw[i], key);
+                    if (mode == STC_MODE_PER_TOKEN) {
+#pragma unroll
+                        for (int j = 0; j < S; ++j) {
+                            int rank = 0;
+#pragma unroll
+                            for (int i2 = 0; i2 < S; ++i2)
+                                rank += (key[i2] > key[j]) || (key[i2] == key[j] && i2 < j);
+                            if (rank < k_nominal) def |= 1u << j;
+                        }
+                    } else {
+                        if (!(flags & FL_NONE)) {
+#pragma unroll
+                            for (int j = 0; j < S; ++j) {
+                                def |= (key[j] > tau ? 1u : 0u) << j;
+                                tie |= (key[j] == tau ? 1u : 0u) << j;
+                            }
+                        }
+                        if (min_per_token) {
+                            const uint32_t bit = 1u << first_max<S>(key);
+                            def |= bit;
+                            tie &= ~bit;
+                        }
+                    }
+                }
+                if (u + i < u0 + n && t < T) {
+                    v_mask[(size_t)problem * T + t] = (uint16_t)def;
+                    tie_all[(size_t)problem * T + t] = (uint16_t)tie;
+                }
+                uint32_t cnt = __popc(def) | (__popc(tie) << 16);   // a unit holds at most 256 * 16 bits of each
+#pragma unroll
+                for (int d = 16; d >= 1; d >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+                if (lane == 0) s_red[i][warp] = cnt;
+            }
+            __syncthreads();
+            if (tid < kBatch && u + tid < u0 + n) {
+                uint32_t tot = 0;
+#pragma unroll
+                for (int w2 = 0; w2 < kWarps; ++w2) tot += s_red[tid][w2];
+                unit_sums[(size_t)problem * upp + u + tid] = tot;
+            }
+            __syncthreads();
+        }
     }
 }
 
 template <int S>
 __global__ void __launch_bounds__(kThreads)
 route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ seq_len, int Hkv, int T,
-                     int n_tiles, int mode, const uint32_t* __restrict__ state_all,
-                     const uint32_t* __restrict__ tile_sums, const uint16_t* __restrict__ tie_all,
+                     int n_tiles, int upp, int mode, const uint32_t* __restrict__ state_all,
+                     const uint32_t* __restrict__ abort_word, const uint32_t* __restrict__ unit_sums,
+                     const uint16_t* __restrict__ tie_all,
                      uint16_t* __restrict__ v_mask, uint32_t* __restrict__ v_offs,
                      uint4* __restrict__ v_packed, int64_t cap_groups, int64_t* __restrict__ total_groups,
                      int32_t* __restrict__ status) {
@@ -362,11 +439,12 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
         flags = __ldcg(state + ST_FLAGS);
         krem = flags ? 0u : __ldcg(state + ST_KREM);
     }
-    // base counts from the preceding tiles
+    // base counts from the preceding units
     uint32_t bd = 0, be = 0;
-    for (int i = tid; i < tile; i += kThreads) {
-        bd += __ldcg(tile_sums + ((size_t)problem * n_tiles + i) * 2 + 0);
-        be += __ldcg(tile_sums + ((size_t)problem * n_tiles + i) * 2 + 1);
+    for (int i = tid; i < tile * kUnitsPerTile; i += kThreads) {
+        const uint32_t c = __ldcg(unit_sums + (size_t)problem * upp + i);
+        bd += c & 0xFFFFu;
+        be += c >> 16;
     }
     uint32_t base_d, base_e;
     block_excl_scan(bd, s_w, &base_d);
@@ -408,7 +486,8 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
             const uint32_t total = len == 0 ? 0u : off + __popc(m);
             v_offs[(size_t)problem * (T + 1) + len] = total;
             total_groups[problem] = (int64_t)total;
-            status[problem] = (flags & FL_BUDGET) ? STC_ERR_BUDGET
+            status[problem] = __ldcg(abort_word) ? STC_ERR_TIMEOUT
+                              : (flags & FL_BUDGET) ? STC_ERR_BUDGET
                               : ((int64_t)total > cap_groups ? STC_ERR_CAPACITY : STC_OK);
         }
     }
@@ -447,6 +526,48 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
 
 size_t route_ws_bytes(const Geom& g) { return carve(g, nullptr).total_bytes; }
 
+namespace {
+
+// CTAs of the select kernel that can be resident at once (it is launched cooperatively).
+template <int S>
+cudaError_t select_grid_limit(int* limit) {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, sms = 0, per_sm = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess)
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, route_select_kernel<S>, kThreads, 0);
+        if (e != cudaSuccess) return e;
+        if (sms <= 0 || per_sm <= 0) return cudaErrorLaunchOutOfResources;
+        cached = sms * per_sm;
+    }
+    *limit = cached;
+    return cudaSuccess;
+}
+
+template <int S>
+cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls, int64_t cls_b, int64_t cls_h,
+                          int k_nominal, int min_per_token, int mode, const RouteWs& w, uint16_t* v_mask,
+                          cudaStream_t st) {
+    int limit = 0;
+    cudaError_t e = select_grid_limit<S>(&limit);
+    if (e != cudaSuccess) return e;
+    int upp = (g.T + kUnit - 1) / kUnit;
+    long long total_units = (long long)upp * g.problems;
+    const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
+    const int32_t* seq_len = g.seq_len;
+    int Hkv = g.Hkv, T = g.T;
+    uint32_t *state = w.state, *hist = w.hist, *abort_word = w.abort_word, *unit_sums = w.unit_sums;
+    uint16_t* tie = w.tie;
+    void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token, &mode,
+                    &state, &hist, &abort_word, &v_mask, &tie, &unit_sums, &total_units};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_select_kernel<S>), dim3(grid),
+                                       dim3(kThreads), args, 0, st);
+}
+
+}  // namespace
+
 cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
                               const uint8_t* tok_class, int64_t class_head_stride, int k_nominal,
                               int min_per_token, int mode, void* v_packed, uint16_t* v_mask,
@@ -456,33 +577,27 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     const RouteWs w = carve(g, ws);
     const bool do_route = phases & 1, do_pack = phases & 2;
     const int n_tiles = (g.T + kTile - 1) / kTile;
+    const int upp = (g.T + kUnit - 1) / kUnit;
     const long long n_cta = (long long)n_tiles * g.problems;
     if (n_cta > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    // score-scanning kernels: enough CTAs for a few waves, several tiles each beyond that
-    int tpc = (int)(n_cta / (148 * 8 * 2));
-    tpc = tpc < 1 ? 1 : (tpc > 16 ? 16 : tpc);
-    const unsigned n_cta_scan = (unsigned)((n_tiles + tpc - 1) / tpc) * (unsigned)g.problems;
     const int64_t cls_h = class_head_stride;
     const int64_t cls_b = class_head_stride ? (int64_t)g.Hkv * class_head_stride : (int64_t)g.T;
+    cudaError_t e = cudaSuccess;
     if (do_route) {
-        cudaError_t e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
+        e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
         if (e != cudaSuccess) return e;
     }
 
 #define STC_ROUTE(S_)                                                                               \
     case S_: {                                                                                      \
-        if (do_route && mode == STC_MODE_GLOBAL)                                                    \
-            for (int pass = 0; pass < 3; ++pass)                                                    \
-                route_hist_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                             \
-                    scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal, \
-                    min_per_token, pass, w.state, w.hist);                                          \
-        if (do_route) route_mask_kernel<S_><<<n_cta_scan, kThreads, 0, st>>>(                                     \
-            scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, n_tiles, tpc, k_nominal,        \
-            min_per_token, mode, w.state, v_mask, w.tie, w.tile_sums);                              \
-        if (do_pack) route_compact_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                             \
-            static_cast<const uint4*>(v), g.seq_len, g.Hkv, g.T, n_tiles, mode, w.state,            \
-            w.tile_sums, w.tie, v_mask, v_offs, static_cast<uint4*>(v_packed), cap_groups,          \
-            total_groups, status);                                                                  \
+        if (do_route)                                                                               \
+            e = launch_select<S_>(g, scores, tok_class, cls_b, cls_h, k_nominal, min_per_token,     \
+                                  mode, w, v_mask, st);                                             \
+        if (e != cudaSuccess) return e;                                                             \
+        if (do_pack) route_compact_kernel<S_><<<(unsigned)n_cta, kThreads, 0, st>>>(                \
+            static_cast<const uint4*>(v), g.seq_len, g.Hkv, g.T, n_tiles, upp, mode, w.state,       \
+            w.abort_word, w.unit_sums, w.tie, v_mask, v_offs, static_cast<uint4*>(v_packed),        \
+            cap_groups, total_groups, status);                                                      \
     } break;
     switch (g.S) {
         STC_ROUTE(4) STC_ROUTE(8) STC_ROUTE(16)
