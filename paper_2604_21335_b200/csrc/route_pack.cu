@@ -47,7 +47,8 @@ struct RouteWs {
     uint32_t* abort_word; // set when a bounded wait gave up
     uint32_t* unit_sums;  // [problems][units]: definite count | tie count << 16
     uint16_t* tie;        // [problems][T]
-    size_t zero_bytes;    // leading bytes (state + hist) cleared per call
+    size_t zero_small;    // leading bytes cleared per call: state and abort word only ...
+    size_t zero_bytes;    // ... or with the global histograms (problems that span several CTAs)
     size_t total_bytes;
 };
 
@@ -59,8 +60,9 @@ RouteWs carve(const Geom& g, void* ws) {
     const int n_units = (g.T + kUnit - 1) / kUnit;
     size_t o = 0;
     r.state = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * ST_WORDS * 4);
-    r.hist = reinterpret_cast<uint32_t*>(p + o);  o += align256((size_t)g.problems * 3 * kBins * 4);
     r.abort_word = reinterpret_cast<uint32_t*>(p + o); o += 256;
+    r.zero_small = o;
+    r.hist = reinterpret_cast<uint32_t*>(p + o);  o += align256((size_t)g.problems * 3 * kBins * 4);
     r.zero_bytes = o;
     r.unit_sums = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * n_units * 4);
     r.tie = reinterpret_cast<uint16_t*>(p + o);   o += align256((size_t)g.problems * g.T * 2);
@@ -135,6 +137,7 @@ __device__ __forceinline__ int token_class(const uint8_t* cls, int t, int len) {
 }
 
 // The last CTA of a pass: find the bin holding the krem-th largest candidate.
+template <bool kSharedHist>
 __device__ void pick_digit(const uint32_t* __restrict__ hist, int nbins, uint32_t krem,
                            uint32_t* s_w, uint32_t* s_out /*[2]: digit, new krem*/) {
     // thread t owns bins nbins-1-8t .. nbins-8-8t (descending); nbins <= 8*kThreads
@@ -142,7 +145,7 @@ __device__ void pick_digit(const uint32_t* __restrict__ hist, int nbins, uint32_
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         int bin = nbins - 1 - 8 * (int)threadIdx.x - j;
-        c[j] = bin >= 0 ? __ldcg(hist + bin) : 0u;
+        c[j] = bin >= 0 ? (kSharedHist ? hist[bin] : __ldcg(hist + bin)) : 0u;
         sum += c[j];
     }
     uint32_t excl = block_excl_scan(sum, s_w, nullptr);
@@ -159,6 +162,62 @@ __device__ void pick_digit(const uint32_t* __restrict__ hist, int nbins, uint32_
         }
     }
     __syncthreads();
+}
+
+// Histogram contribution of one routed token in one pass: its keys that still match the
+// resolved prefix, except the reserved first maximum.
+template <int S>
+__device__ __forceinline__ void hist_token(const uint32_t (&key)[S], uint32_t himask, uint32_t prefix, int dshift,
+                                           uint32_t dmask, int min_per_token, uint32_t* shist) {
+    uint32_t cand = 0;
+#pragma unroll
+    for (int j = 0; j < S; ++j) cand |= ((key[j] & himask) == prefix ? 1u : 0u) << j;
+    if (cand == 0u) return;
+    if (min_per_token) cand &= ~(1u << first_max<S>(key));
+#pragma unroll
+    for (int j = 0; j < S; ++j)
+        if ((cand >> j) & 1u) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
+}
+
+// Definite and tie bits of one routed token against the final threshold.
+template <int S>
+__device__ __forceinline__ void mask_token(const uint32_t (&key)[S], int mode, uint32_t flags, uint32_t tau,
+                                           int k_nominal, int min_per_token, uint32_t& def, uint32_t& tie) {
+    def = 0;
+    tie = 0;
+    if (mode == STC_MODE_PER_TOKEN) {
+#pragma unroll
+        for (int j = 0; j < S; ++j) {
+            int rank = 0;
+#pragma unroll
+            for (int i2 = 0; i2 < S; ++i2) rank += (key[i2] > key[j]) || (key[i2] == key[j] && i2 < j);
+            if (rank < k_nominal) def |= 1u << j;
+        }
+        return;
+    }
+    if (!(flags & FL_NONE)) {
+#pragma unroll
+        for (int j = 0; j < S; ++j) {
+            def |= (key[j] > tau ? 1u : 0u) << j;
+            tie |= (key[j] == tau ? 1u : 0u) << j;
+        }
+    }
+    if (min_per_token) {
+        const uint32_t bit = 1u << first_max<S>(key);
+        def |= bit;
+        tie &= ~bit;
+    }
+}
+
+// Budget of a problem from its routed-token count: flags (FL_*) and the number of pairs to
+// take beyond the reserved ones.
+__device__ __forceinline__ uint32_t budget_of(uint64_t n_routed, int k_nominal, int min_per_token, uint32_t& flags) {
+    const uint64_t m_total = n_routed * (uint64_t)k_nominal;
+    flags = 0;
+    if (min_per_token && m_total < n_routed) flags = FL_BUDGET;
+    const uint64_t take = m_total - (min_per_token ? n_routed : 0);
+    if (!flags && take == 0) flags = FL_NONE;
+    return (uint32_t)take;
 }
 
 // ---- bounded cross-CTA hand-off -------------------------------------------------
@@ -273,14 +332,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
                     ++n_routed;
                     uint32_t key[S];
                     make_keys<S>(raw[i], key);
-                    uint32_t cand = 0;                   // keys still in the running for this pass
-#pragma unroll
-                    for (int j = 0; j < S; ++j) cand |= ((key[j] & himask) == prefix ? 1u : 0u) << j;
-                    if (cand == 0u) continue;
-                    if (min_per_token) cand &= ~(1u << first_max<S>(key));
-#pragma unroll
-                    for (int j = 0; j < S; ++j)
-                        if ((cand >> j) & 1u) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
+                    hist_token<S>(key, himask, prefix, dshift, dmask, min_per_token, shist);
                 }
             }
             __syncthreads();
@@ -304,17 +356,12 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             // the CTA that completed the problem's pass picks the digit and publishes it
             uint32_t krem = krem_in, flags = 0;
             if (pass == 0) {
-                const uint64_t nr = __ldcg(state + ST_NROUTED);
-                const uint64_t m_total = nr * (uint64_t)k_nominal;
-                if (min_per_token && m_total < nr) flags = FL_BUDGET;
-                const uint64_t take = m_total - (min_per_token ? nr : 0);
-                if (!flags && take == 0) flags = FL_NONE;
-                krem = (uint32_t)take;
+                krem = budget_of(__ldcg(state + ST_NROUTED), k_nominal, min_per_token, flags);
             }
             if (flags) {
                 if (tid == 0) { state[ST_FLAGS] = flags; state[ST_PREFIX] = 0; state[ST_KREM] = 0; }
             } else {
-                pick_digit(hist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
+                pick_digit<false>(hist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
                 if (tid == 0) {
                     state[ST_PREFIX] = prefix | (s_pick[0] << pass_shift(pass));
                     state[ST_KREM] = s_pick[1];
@@ -366,29 +413,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
                 } else if (cl == STC_CLS_ROUTED) {
                     uint32_t key[S];
                     make_keys<S>(raw[i], key);
-                    if (mode == STC_MODE_PER_TOKEN) {
-#pragma unroll
-                        for (int j = 0; j < S; ++j) {
-                            int rank = 0;
-#pragma unroll
-                            for (int i2 = 0; i2 < S; ++i2)
-                                rank += (key[i2] > key[j]) || (key[i2] == key[j] && i2 < j);
-                            if (rank < k_nominal) def |= 1u << j;
-                        }
-                    } else {
-                        if (!(flags & FL_NONE)) {
-#pragma unroll
-                            for (int j = 0; j < S; ++j) {
-                                def |= (key[j] > tau ? 1u : 0u) << j;
-                                tie |= (key[j] == tau ? 1u : 0u) << j;
-                            }
-                        }
-                        if (min_per_token) {
-                            const uint32_t bit = 1u << first_max<S>(key);
-                            def |= bit;
-                            tie &= ~bit;
-                        }
-                    }
+                    mask_token<S>(key, mode, flags, tau, k_nominal, min_per_token, def, tie);
                 }
                 if (u + i < u0 + n && t < T) {
                     v_mask[(size_t)problem * T + t] = (uint16_t)def;
@@ -408,6 +433,106 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             }
             __syncthreads();
         }
+    }
+}
+
+// Problems of at most kBatch units (one token per thread and unit): a CTA takes whole
+// problems, keeps their keys in registers and resolves the three digits from its own
+// shared-memory histogram -- no global histogram, no hand-off between CTAs.
+template <int S>
+__global__ void __launch_bounds__(kThreads)
+route_select_small_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls,
+                          int64_t cls_b_stride, int64_t cls_h_stride, const int32_t* __restrict__ seq_len,
+                          int Hkv, int T, int upp, int k_nominal, int min_per_token, int mode,
+                          uint32_t* __restrict__ state_all, uint16_t* __restrict__ v_mask,
+                          uint16_t* __restrict__ tie_all, uint32_t* __restrict__ unit_sums, int problems) {
+    constexpr int kBatch = 32 / S;
+    __shared__ uint32_t shist[kBins];
+    __shared__ uint32_t s_w[kWarps];
+    __shared__ uint32_t s_red[kBatch][kWarps];
+    __shared__ uint32_t s_pick[2];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+#pragma unroll 1
+    for (int problem = blockIdx.x; problem < problems; problem += gridDim.x) {
+        const int b = problem / Hkv, hk = problem - b * Hkv;
+        const int len = clamp_len(seq_len, b, T);
+        const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+        uint4 raw[kBatch][S / 4];
+        int cls_of[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int t = i * kUnit + tid;
+            cls_of[i] = (i < upp && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
+            if (cls_of[i] == STC_CLS_ROUTED) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+        }
+        uint32_t key[kBatch][S];
+        uint32_t n_routed = 0;
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            if (cls_of[i] == STC_CLS_ROUTED) {
+                make_keys<S>(raw[i], key[i]);
+                ++n_routed;
+            } else {
+#pragma unroll
+                for (int j = 0; j < S; ++j) key[i][j] = 0u;
+            }
+        }
+        uint32_t tau = 0, flags = 0, krem = 0;
+        if (mode == STC_MODE_GLOBAL) {
+            uint32_t tot;
+            block_excl_scan(n_routed, s_w, &tot);
+            krem = budget_of(tot, k_nominal, min_per_token, flags);
+#pragma unroll 1
+            for (int pass = 0; pass < 3 && !flags; ++pass) {
+                for (int i = tid; i < kBins; i += kThreads) shist[i] = 0;
+                __syncthreads();
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i)
+                    if (cls_of[i] == STC_CLS_ROUTED)
+                        hist_token<S>(key[i], pass_himask(pass), tau, pass_shift(pass), pass == 2 ? 1023u : 2047u,
+                                      min_per_token, shist);
+                __syncthreads();
+                pick_digit<true>(shist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
+                tau |= s_pick[0] << pass_shift(pass);
+                krem = s_pick[1];
+                __syncthreads();                       // s_pick and the histogram are reused by the next pass
+            }
+            if (tid == 0) {                            // what the compaction kernel reads
+                uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+                state[ST_FLAGS] = flags;
+                state[ST_PREFIX] = flags ? 0u : tau;
+                state[ST_KREM] = flags ? 0u : krem;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int t = i * kUnit + tid;
+            uint32_t def = 0, tie = 0;
+            if (flags & FL_BUDGET) {
+                def = 0;
+            } else if (cls_of[i] == STC_CLS_FULL) {
+                def = (1u << S) - 1u;
+            } else if (cls_of[i] == STC_CLS_ROUTED) {
+                mask_token<S>(key[i], mode, flags, tau, k_nominal, min_per_token, def, tie);
+            }
+            if (i < upp && t < T) {
+                v_mask[(size_t)problem * T + t] = (uint16_t)def;
+                tie_all[(size_t)problem * T + t] = (uint16_t)tie;
+            }
+            uint32_t cnt = __popc(def) | (__popc(tie) << 16);
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+            if (lane == 0) s_red[i][warp] = cnt;
+        }
+        __syncthreads();
+        if (tid < kBatch && tid < upp) {
+            uint32_t tot = 0;
+#pragma unroll
+            for (int w2 = 0; w2 < kWarps; ++w2) tot += s_red[tid][w2];
+            unit_sums[(size_t)problem * upp + tid] = tot;
+        }
+        __syncthreads();
     }
 }
 
@@ -583,14 +708,20 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     const int64_t cls_h = class_head_stride;
     const int64_t cls_b = class_head_stride ? (int64_t)g.Hkv * class_head_stride : (int64_t)g.T;
     cudaError_t e = cudaSuccess;
+    const bool small = upp <= 32 / g.S;            // a problem fits one CTA's registers
     if (do_route) {
-        e = cudaMemsetAsync(w.state, 0, w.zero_bytes, st);
+        e = cudaMemsetAsync(w.state, 0, small ? w.zero_small : w.zero_bytes, st);
         if (e != cudaSuccess) return e;
     }
+    const unsigned grid_small = (unsigned)(g.problems < 148 * 16 ? g.problems : 148 * 16);
 
 #define STC_ROUTE(S_)                                                                               \
     case S_: {                                                                                      \
-        if (do_route)                                                                               \
+        if (do_route && small)                                                                      \
+            route_select_small_kernel<S_><<<grid_small, kThreads, 0, st>>>(                         \
+                scores, tok_class, cls_b, cls_h, g.seq_len, g.Hkv, g.T, upp, k_nominal,             \
+                min_per_token, mode, w.state, v_mask, w.tie, w.unit_sums, g.problems);              \
+        else if (do_route)                                                                          \
             e = launch_select<S_>(g, scores, tok_class, cls_b, cls_h, k_nominal, min_per_token,     \
                                   mode, w, v_mask, st);                                             \
         if (e != cudaSuccess) return e;                                                             \
