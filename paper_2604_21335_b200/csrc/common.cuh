@@ -64,12 +64,15 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr) {
     return r;
 }
 
-// Order-preserving map from fp32 bits to uint32 (larger float -> larger key);
-// -0 is folded onto +0 so the two compare equal.
+// Order-preserving map from fp32 to uint32 (larger float -> larger key); -0 is folded
+// onto +0 (by the addition) so the two compare equal.
 __device__ __forceinline__ uint32_t float_key(float f) {
-    const uint32_t u = __float_as_uint(f);
-    const uint32_t k = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);   // negative: ~u, else u | sign
-    return k + (k == 0x7FFFFFFFu);                                          // -0 (0x7FFFFFFF) joins +0 (0x80000000)
+    const uint32_t u = __float_as_uint(__fadd_rn(f, 0.0f));
+    return u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);               // negative: ~u, else u | sign
+}
+// The float whose key is k (k = 0x7FFFFFFF, the unused key of -0, gives -0).
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
 // ---- internal launchers (one per source file) -------------------------------

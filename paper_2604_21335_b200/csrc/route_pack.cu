@@ -164,19 +164,49 @@ __device__ void pick_digit(const uint32_t* __restrict__ hist, int nbins, uint32_
     __syncthreads();
 }
 
+template <int S>
+__device__ __forceinline__ uint32_t max_key(const uint32_t (&key)[S]) {
+    uint32_t m = key[0];
+#pragma unroll
+    for (int j = 1; j + 1 < S; j += 2) m = max(m, max(key[j], key[j + 1]));
+    return max(m, key[S - 1]);
+}
+
 // Histogram contribution of one routed token in one pass: its keys that still match the
-// resolved prefix, except the reserved first maximum.
+// resolved prefix, except the reserved first maximum (counted, then taken back: equal
+// keys share a bin, so which of them is the reserved one does not matter here).
 template <int S>
 __device__ __forceinline__ void hist_token(const uint32_t (&key)[S], uint32_t himask, uint32_t prefix, int dshift,
                                            uint32_t dmask, int min_per_token, uint32_t* shist) {
-    uint32_t cand = 0;
-#pragma unroll
-    for (int j = 0; j < S; ++j) cand |= ((key[j] & himask) == prefix ? 1u : 0u) << j;
-    if (cand == 0u) return;
-    if (min_per_token) cand &= ~(1u << first_max<S>(key));
 #pragma unroll
     for (int j = 0; j < S; ++j)
-        if ((cand >> j) & 1u) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
+        if ((key[j] & himask) == prefix) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
+    if (min_per_token) {
+        const uint32_t bk = max_key<S>(key);
+        if ((bk & himask) == prefix) atomicSub(&shist[(bk >> dshift) & dmask], 1u);
+    }
+}
+
+// Bounds, as floats, of the keys that match a resolved prefix: lo <= x <= hi is what the
+// later passes test before they build any key (scores are not NaN).
+__device__ __forceinline__ void prefix_bounds(uint32_t prefix, uint32_t himask, float& lo, float& hi) {
+    uint32_t klo = prefix, khi = prefix | ~himask;
+    klo = max(klo, 0x007FFFFFu);                   // -inf
+    khi = min(khi, 0xFF800000u);                   // +inf
+    if (khi == 0x7FFFFFFFu) khi = 0x7FFFFFFEu;     // the key of -0 is unused: stop below zero
+    lo = key_float(klo);
+    hi = key_float(khi);
+}
+template <int S>
+__device__ __forceinline__ bool any_in_bounds(const uint4 (&raw)[S / 4], float lo, float hi) {
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < S / 4; ++i) {
+        const float x0 = __uint_as_float(raw[i].x), x1 = __uint_as_float(raw[i].y);
+        const float x2 = __uint_as_float(raw[i].z), x3 = __uint_as_float(raw[i].w);
+        any |= (x0 >= lo && x0 <= hi) || (x1 >= lo && x1 <= hi) || (x2 >= lo && x2 <= hi) || (x3 >= lo && x3 <= hi);
+    }
+    return any;
 }
 
 // Definite and tie bits of one routed token against the final threshold.
@@ -202,9 +232,13 @@ __device__ __forceinline__ void mask_token(const uint32_t (&key)[S], int mode, u
             tie |= (key[j] == tau ? 1u : 0u) << j;
         }
     }
-    if (min_per_token) {
-        const uint32_t bit = 1u << first_max<S>(key);
-        def |= bit;
+    if (min_per_token && def == 0u) {
+        // The reserved group is the token's first maximum.  With a key above the threshold it is
+        // among the definite bits already; with the maximum on the threshold it is the first tie.
+        uint32_t bit;
+        if (tie) bit = tie & (0u - tie);
+        else bit = 1u << first_max<S>(key);
+        def = bit;
         tie &= ~bit;
     }
 }
@@ -303,6 +337,18 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             const int len = clamp_len(seq_len, b, T);
             uint32_t* state = state_all + (size_t)problem * ST_WORDS;
             uint32_t* hist = hist_all + ((size_t)problem * 3 + pass) * kBins;
+            const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+            uint4 raw[kBatch][S / 4];
+            bool routed[kBatch];
+            auto load_batch = [&](int u) {               // all of the thread's loads are in flight before the first use
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) {
+                    const int t = (u + i) * kUnit + tid;
+                    routed[i] = u + i < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
+                    if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+                }
+            };
+            load_batch(u0);                              // in flight while the digit of the previous pass arrives
             uint32_t prefix = 0, krem_in = 0;
             if (pass > 0) {
                 if (!wait_done(state, (uint32_t)pass, s_bc, abort_word)) return;
@@ -312,24 +358,19 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             }
             for (int i = tid; i < kBins; i += kThreads) shist[i] = 0;
             __syncthreads();
+            float lo, hi;
+            prefix_bounds(prefix, himask, lo, hi);
 
-            const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
             uint32_t n_routed = 0;
 #pragma unroll 1
             for (int u = u0; u < u0 + n; u += kBatch) {
                 if (u * kUnit >= len) break;
-                uint4 raw[kBatch][S / 4];                // all of the thread's loads are in flight before the first use
-                bool routed[kBatch];
-#pragma unroll
-                for (int i = 0; i < kBatch; ++i) {
-                    const int t = (u + i) * kUnit + tid;
-                    routed[i] = u + i < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
-                    if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
-                }
+                if (u != u0) load_batch(u);
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) {
                     if (!routed[i]) continue;
                     ++n_routed;
+                    if (pass > 0 && !any_in_bounds<S>(raw[i], lo, hi)) continue;
                     uint32_t key[S];
                     make_keys<S>(raw[i], key);
                     hist_token<S>(key, himask, prefix, dshift, dmask, min_per_token, shist);
@@ -384,6 +425,17 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
         const int b = problem / Hkv, hk = problem - b * Hkv;
         const int len = clamp_len(seq_len, b, T);
         const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+        uint4 raw[kBatch][S / 4];
+        int cls_of[kBatch];
+        auto load_batch = [&](int u) {
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int t = (u + i) * kUnit + tid;
+                cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
+                if (cls_of[i] == STC_CLS_ROUTED) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+            }
+        };
+        load_batch(u0);                                  // in flight while the last digit arrives
         uint32_t tau = 0, flags = 0;
         if (mode == STC_MODE_GLOBAL) {
             if (!wait_done(state_all + (size_t)problem * ST_WORDS, 3u, s_bc, abort_word)) return;
@@ -392,15 +444,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
         }
 #pragma unroll 1
         for (int u = u0; u < u0 + n; u += kBatch) {
-            uint4 raw[kBatch][S / 4];
-            int cls_of[kBatch];
-#pragma unroll
-            for (int i = 0; i < kBatch; ++i) {
-                const int t = (u + i) * kUnit + tid;
-                cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
-                if (cls_of[i] == STC_CLS_ROUTED && !(flags & FL_BUDGET))
-                    load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
-            }
+            if (u != u0) load_batch(u);
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
                 const int t = (u + i) * kUnit + tid;
