@@ -172,18 +172,29 @@ __device__ __forceinline__ uint32_t max_key(const uint32_t (&key)[S]) {
     return max(m, key[S - 1]);
 }
 
+// shist[bin] += delta when `on` (a predicated reduction: no branch per key).
+__device__ __forceinline__ void red_if(bool on, uint32_t shist_base, uint32_t bin, int delta) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p red.shared.add.u32 [%1], %2;\n\t}"
+        ::"r"((uint32_t)on), "r"(shist_base + bin * 4u), "r"((uint32_t)delta) : "memory");
+}
+
 // Histogram contribution of one routed token in one pass: its keys that still match the
 // resolved prefix, except the reserved first maximum (counted, then taken back: equal
 // keys share a bin, so which of them is the reserved one does not matter here).
-template <int S>
+template <int S, bool kFirstPass>
 __device__ __forceinline__ void hist_token(const uint32_t (&key)[S], uint32_t himask, uint32_t prefix, int dshift,
-                                           uint32_t dmask, int min_per_token, uint32_t* shist) {
+                                           uint32_t dmask, int min_per_token, uint32_t shist_base) {
+    const uint32_t bk = max_key<S>(key);
+    if (kFirstPass) {                              // every key is a candidate; the digit is the top 11 bits
 #pragma unroll
-    for (int j = 0; j < S; ++j)
-        if ((key[j] & himask) == prefix) atomicAdd(&shist[(key[j] >> dshift) & dmask], 1u);
-    if (min_per_token) {
-        const uint32_t bk = max_key<S>(key);
-        if ((bk & himask) == prefix) atomicSub(&shist[(bk >> dshift) & dmask], 1u);
+        for (int j = 0; j < S; ++j) red_if(true, shist_base, key[j] >> 21, 1);
+        red_if(min_per_token != 0, shist_base, bk >> 21, -1);
+    } else {
+#pragma unroll
+        for (int j = 0; j < S; ++j)
+            red_if((key[j] & himask) == prefix, shist_base, (key[j] >> dshift) & dmask, 1);
+        red_if(min_per_token != 0 && (bk & himask) == prefix, shist_base, (bk >> dshift) & dmask, -1);
     }
 }
 
@@ -226,10 +237,15 @@ __device__ __forceinline__ void mask_token(const uint32_t (&key)[S], int mode, u
         return;
     }
     if (!(flags & FL_NONE)) {
+        bool any_tie = false;
 #pragma unroll
         for (int j = 0; j < S; ++j) {
             def |= (key[j] > tau ? 1u : 0u) << j;
-            tie |= (key[j] == tau ? 1u : 0u) << j;
+            any_tie |= key[j] == tau;
+        }
+        if (any_tie) {
+#pragma unroll
+            for (int j = 0; j < S; ++j) tie |= (key[j] == tau ? 1u : 0u) << j;
         }
     }
     if (min_per_token && def == 0u) {
@@ -340,12 +356,13 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
             uint4 raw[kBatch][S / 4];
             bool routed[kBatch];
+            const float* rows = scores + (size_t)problem * T * S;
             auto load_batch = [&](int u) {               // all of the thread's loads are in flight before the first use
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) {
                     const int t = (u + i) * kUnit + tid;
                     routed[i] = u + i < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
-                    if (routed[i]) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+                    load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);   // unconditional: no branch per token
                 }
             };
             load_batch(u0);                              // in flight while the digit of the previous pass arrives
@@ -360,20 +377,32 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             __syncthreads();
             float lo, hi;
             prefix_bounds(prefix, himask, lo, hi);
+            const uint32_t shist_base = smem_u32(shist);
 
             uint32_t n_routed = 0;
 #pragma unroll 1
             for (int u = u0; u < u0 + n; u += kBatch) {
                 if (u * kUnit >= len) break;
                 if (u != u0) load_batch(u);
+                if (pass == 0) {
 #pragma unroll
-                for (int i = 0; i < kBatch; ++i) {
-                    if (!routed[i]) continue;
-                    ++n_routed;
-                    if (pass > 0 && !any_in_bounds<S>(raw[i], lo, hi)) continue;
-                    uint32_t key[S];
-                    make_keys<S>(raw[i], key);
-                    hist_token<S>(key, himask, prefix, dshift, dmask, min_per_token, shist);
+                    for (int i = 0; i < kBatch; ++i) {
+                        n_routed += routed[i];
+                        if (routed[i]) {
+                            uint32_t key[S];
+                            make_keys<S>(raw[i], key);
+                            hist_token<S, true>(key, 0u, 0u, 21, 2047u, min_per_token, shist_base);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i) {
+                        if (routed[i] && any_in_bounds<S>(raw[i], lo, hi)) {
+                            uint32_t key[S];
+                            make_keys<S>(raw[i], key);
+                            hist_token<S, false>(key, himask, prefix, dshift, dmask, min_per_token, shist_base);
+                        }
+                    }
                 }
             }
             __syncthreads();
@@ -427,12 +456,13 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
         const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
         uint4 raw[kBatch][S / 4];
         int cls_of[kBatch];
+        const float* rows = scores + (size_t)problem * T * S;
         auto load_batch = [&](int u) {
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
                 const int t = (u + i) * kUnit + tid;
                 cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
-                if (cls_of[i] == STC_CLS_ROUTED) load_raw<S>(scores + ((size_t)problem * T + t) * S, raw[i]);
+                load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);
             }
         };
         load_batch(u0);                                  // in flight while the last digit arrives
@@ -463,9 +493,8 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
                     v_mask[(size_t)problem * T + t] = (uint16_t)def;
                     tie_all[(size_t)problem * T + t] = (uint16_t)tie;
                 }
-                uint32_t cnt = __popc(def) | (__popc(tie) << 16);   // a unit holds at most 256 * 16 bits of each
-#pragma unroll
-                for (int d = 16; d >= 1; d >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+                // a unit holds at most 256 * 16 bits of each kind: both counts fit one word
+                const uint32_t cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(def) | (__popc(tie) << 16));
                 if (lane == 0) s_red[i][warp] = cnt;
             }
             __syncthreads();
@@ -534,8 +563,8 @@ route_select_small_kernel(const float* __restrict__ scores, const uint8_t* __res
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i)
                     if (cls_of[i] == STC_CLS_ROUTED)
-                        hist_token<S>(key[i], pass_himask(pass), tau, pass_shift(pass), pass == 2 ? 1023u : 2047u,
-                                      min_per_token, shist);
+                        hist_token<S, false>(key[i], pass_himask(pass), tau, pass_shift(pass),
+                                             pass == 2 ? 1023u : 2047u, min_per_token, smem_u32(shist));
                 __syncthreads();
                 pick_digit<true>(shist, pass == 2 ? 1024 : kBins, krem, s_w, s_pick);
                 tau |= s_pick[0] << pass_shift(pass);
@@ -564,9 +593,7 @@ route_select_small_kernel(const float* __restrict__ scores, const uint8_t* __res
                 v_mask[(size_t)problem * T + t] = (uint16_t)def;
                 tie_all[(size_t)problem * T + t] = (uint16_t)tie;
             }
-            uint32_t cnt = __popc(def) | (__popc(tie) << 16);
-#pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, d);
+            const uint32_t cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(def) | (__popc(tie) << 16));
             if (lane == 0) s_red[i][warp] = cnt;
         }
         __syncthreads();
