@@ -176,8 +176,12 @@ int32_t stc_quest_select_static(const stc_shape* shape, const stc_cache* cache, 
  *   (ties to the lower group).
  * Outputs: out->v_mask (0 for tokens past len), out->v_offs[0..len],
  * out->v_packed, total_groups i64 [B][Hkv], status i32 [B][Hkv] (STC_OK,
- * STC_ERR_BUDGET: nothing packed for that problem, or STC_ERR_CAPACITY: groups
- * past cap_groups were not stored).  Non-finite scores are not supported.
+ * STC_ERR_BUDGET: nothing packed for that problem, STC_ERR_CAPACITY: groups
+ * past cap_groups were not stored, or STC_ERR_TIMEOUT in every entry: a
+ * bounded wait between the CTAs of the selection kernel expired and the masks
+ * are not valid; all writes stay in bounds).  Non-finite scores are not
+ * supported.  The selection kernel is launched cooperatively (its whole grid
+ * is resident), so the device must support cooperative launches.
  * ws: STC_OP_ROUTE_PACK. */
 int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* scores,
                        const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
