@@ -30,7 +30,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kTile = 1024;                   // tokens per CTA of the compaction kernel
+constexpr int kTile = 512;                    // tokens per CTA of the compaction kernel
 constexpr int kUnit = kThreads;               // tokens per unit of the score scans (one per thread)
 constexpr int kUnitsPerTile = kTile / kUnit;
 constexpr int kTokPerThread = kTile / kThreads;
@@ -608,7 +608,7 @@ route_select_small_kernel(const float* __restrict__ scores, const uint8_t* __res
 }
 
 template <int S>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ seq_len, int Hkv, int T,
                      int n_tiles, int upp, int mode, const uint32_t* __restrict__ state_all,
                      const uint32_t* __restrict__ abort_word, const uint32_t* __restrict__ unit_sums,
@@ -646,7 +646,7 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
     block_excl_scan(bd, s_w, &base_d);
     block_excl_scan(be, s_w, &base_e);
 
-    // four consecutive tokens per thread keep the scan in token order
+    // consecutive tokens per thread keep the scan in token order
     const int t0 = t_begin + tid * kTokPerThread;
     uint32_t def[kTokPerThread], tie[kTokPerThread], nd = 0, ne = 0;
 #pragma unroll
