@@ -258,3 +258,16 @@ def router_logits(h, w, S, bias=None):
                               _p(np.ascontiguousarray(h), np.uint16), _p(np.ascontiguousarray(w), np.uint16),
                               _p(b), _p(out))
     return out
+
+
+def query_bias(h_q, w_q, q_len=None):
+    """h_q uint16 [B,Lq,d_model], w_q uint16 [N,d_model], q_len int32 [B] or None -> (s_q f64 [B,d_model], bias f64 [B,N])."""
+    B, Lq, dm = h_q.shape
+    N = w_q.shape[0]
+    s_q = np.zeros((B, dm), np.float64)
+    bias = np.zeros((B, N), np.float64)
+    ql = None if q_len is None else np.ascontiguousarray(q_len, np.int32)
+    lib().stc_o_query_bias(C.c_int32(B), C.c_int32(Lq), C.c_int32(dm), C.c_int32(N),
+                           _p(np.ascontiguousarray(h_q), np.uint16), _p(ql),
+                           _p(np.ascontiguousarray(w_q), np.uint16), _p(s_q), _p(bias))
+    return s_q, bias

@@ -502,6 +502,38 @@ void stc_o_router_logits(int32_t B, int32_t Hkv, int32_t T, int32_t S, int32_t d
     }
 }
 
+/* ----------------------------------------------------------------------
+ * Query summary and its router term (Section 3.4: the router sees the token's
+ * hidden state and a summary s_Q of the query region; the summary operator and
+ * g are not specified, the reading taken here is s_Q = mean of the query-region
+ * hidden states and g linear in [h ; s_Q], so the query enters as one additive
+ * term per sequence):
+ *     s_q[b][c]  = (1 / q_len[b]) * sum_{t < q_len[b]} h_q[b][t][c]     (0 when q_len[b] = 0)
+ *     bias[b][n] = sum_c s_q[b][c] * w_q[n][c]
+ *   h_q   [B][Lq][d_model] bf16 bits, q_len [B] or NULL (= Lq), w_q [N][d_model] bf16 bits
+ *   s_q   [B][d_model] fp64, bias [B][N] fp64
+ * ---------------------------------------------------------------------- */
+void stc_o_query_bias(int32_t B, int32_t Lq, int32_t d_model, int32_t N, const uint16_t* h_q,
+                      const int32_t* q_len, const uint16_t* w_q, double* s_q, double* bias) {
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t n_tok = q_len ? q_len[b] : Lq;
+        if (n_tok < 0) n_tok = 0;
+        if (n_tok > Lq) n_tok = Lq;
+        for (int32_t c = 0; c < d_model; ++c) {
+            double acc = 0.0;
+            for (int32_t t = 0; t < n_tok; ++t)
+                acc += (double)bf16_to_f32(h_q[((size_t)b * Lq + t) * d_model + c]);
+            s_q[(size_t)b * d_model + c] = n_tok > 0 ? acc / (double)n_tok : 0.0;
+        }
+        for (int32_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int32_t c = 0; c < d_model; ++c)
+                acc += s_q[(size_t)b * d_model + c] * (double)bf16_to_f32(w_q[(size_t)n * d_model + c]);
+            bias[(size_t)b * N + n] = acc;
+        }
+    }
+}
+
 int32_t stc_o_max_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

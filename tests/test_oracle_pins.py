@@ -451,3 +451,41 @@ def test_batched_drivers_agree_with_single_problem_calls():
                 o1, l1 = O.attend_packed(qg[j], k[b, hk], pk, mk, of, L, w.n_groups, sel, SCALE)
                 np.testing.assert_array_equal(out[b, hk * w.gq + j], o1)
                 assert lse[b, hk * w.gq + j] == l1
+
+
+# ---------------------------------------------------------------------- query summary term
+def test_query_bias_hand_example_constant_rows_and_empty_region():
+    # hand-worked: two query tokens (1, 3) and (3, 5): mean (2, 4); rows (1, -1) -> -2 and (0.5, 0.5) -> 3
+    h = bf16(torch.tensor([[[1.0, 3.0], [3.0, 5.0]]]))
+    w = bf16(torch.tensor([[1.0, -1.0], [0.5, 0.5]]))
+    s_q, bias = O.query_bias(h, w)
+    np.testing.assert_array_equal(s_q, [[2.0, 4.0]])
+    np.testing.assert_array_equal(bias, [[-2.0, 3.0]])
+    # the same rows repeated: the mean is the row itself, one-hot weights pick its channels;
+    # a sequence with an empty query region contributes nothing
+    g = rng(22)
+    row = bf16(torch.randn(3, 1, 32, generator=g))
+    hq = np.repeat(row, 7, axis=1)
+    wq = np.zeros((4, 32), np.uint16)
+    one = bf16(torch.tensor([1.0]))[0]
+    for n, c in enumerate([5, 0, 31, 5]):
+        wq[n, c] = one
+    s_q, bias = O.query_bias(hq, wq, np.array([7, 3, 0], np.int32))
+    np.testing.assert_array_equal(s_q[:2], f32(row)[:2, 0].astype(np.float64))
+    np.testing.assert_array_equal(bias[:2], f32(row)[:2, 0][:, [5, 0, 31, 5]].astype(np.float64))
+    assert not s_q[2].any() and not bias[2].any()
+
+
+def test_query_bias_is_the_mean_of_the_per_token_logits():
+    # linearity: W s_Q = mean_t (W h_t); the per-token logits come from the router pinned above
+    g = rng(23)
+    B, Lq, dm, Hkv, S = 3, 11, 64, 2, 4
+    hq = bf16(torch.randn(B, Lq, dm, generator=g))
+    wq = bf16(torch.randn(Hkv * S, dm, generator=g))
+    q_len = np.array([11, 4, 1], np.int32)
+    s_q, bias = O.query_bias(hq, wq, q_len)
+    per_tok = O.router_logits(hq, wq, S)                      # [B, Hkv, Lq, S]
+    for b in range(B):
+        want = per_tok[b, :, : q_len[b], :].mean(axis=1).reshape(-1)
+        np.testing.assert_allclose(bias[b], want, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(s_q[b], f32(hq)[b, : q_len[b]].astype(np.float64).mean(axis=0), rtol=0, atol=1e-14)
