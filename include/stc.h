@@ -223,6 +223,23 @@ int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, con
 int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, const float* bias_opt,
                           int32_t d_model, float* scores, int32_t* status_word, void* stream);
 
+/* Query summary and its router term (Section 3.4 "query-aware routing": the
+ * router sees the token's hidden state and a summary s_Q of the query region;
+ * the paper fixes neither the summary operator nor g -- taken here: s_Q = mean
+ * of the query-region hidden states, g linear in [h ; s_Q], so the query adds
+ * one term per sequence and logit, the bias_opt of stc_router_logits):
+ *     s_q[b][c]  = (1 / len_b) * sum_{t < len_b} h_q[b][t][c]     (0 when len_b = 0)
+ *     bias[b][n] = sum_c s_q[b][c] * w_q[n][c]
+ *   h_q        bf16 [batch][q_cap][d_model]   hidden states of the query region
+ *   q_len_opt  i32  [batch] or NULL (= q_cap); clamped to 0..q_cap
+ *   w_q        bf16 [n_logits][d_model]       the s_Q half of the router weights
+ *   s_q        f32  [batch][d_model]  (out)    bias  f32 [batch][n_logits]  (out)
+ * fp32 accumulation in a fixed order (repeatable bit for bit).  d_model must be
+ * a multiple of 8 (else STC_ERR_UNSUPPORTED), batch <= 65535; h_q, w_q, s_q
+ * 16-byte aligned; all pointers are device pointers.  Needs no workspace. */
+int32_t stc_query_bias(int32_t batch, int32_t q_cap, int32_t d_model, int32_t n_logits, const void* h_q,
+                       const int32_t* q_len_opt, const void* w_q, float* s_q, float* bias, void* stream);
+
 /* Streaming append (Section 3.4: "query-region tokens are not compressed" -- the
  * tokens generated during decoding keep their full values).  For every sequence
  * b the tokens old_len[b] <= t < len[b] (len = shape->seq_len AFTER the append,

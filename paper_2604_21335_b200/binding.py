@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias",
 )
 
 
@@ -81,6 +81,8 @@ def load_library():
                                         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_append_tokens.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.stc_query_bias.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_router_logits.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_decode_attn.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_void_p,
@@ -266,6 +268,16 @@ def router_logits(shape: Shape, h: torch.Tensor, w: torch.Tensor, scores: torch.
         C.byref(cs), _ptr(h, torch.bfloat16, "h"), _ptr(w, torch.bfloat16, "w"), _ptr(bias, torch.float32, "bias"),
         h.shape[-1], _ptr(scores, torch.float32, "scores"), _ptr(status_word, torch.int32, "status_word"),
         _stream()), "stc_router_logits")
+
+
+def query_bias(h_q: torch.Tensor, w_q: torch.Tensor, s_q: torch.Tensor, bias: torch.Tensor,
+               q_len: Optional[torch.Tensor] = None) -> None:
+    """s_q[b,:] = mean of h_q[b,:q_len[b],:]; bias[b,n] = s_q[b,:] . w_q[n,:]; h_q bf16 [B,Lq,d_model], w_q bf16 [N,d_model]."""
+    B, Lq, dm = h_q.shape
+    _check(load_library().stc_query_bias(
+        B, Lq, dm, w_q.shape[0], _ptr(h_q, torch.bfloat16, "h_q"), _ptr(q_len, torch.int32, "q_len"),
+        _ptr(w_q, torch.bfloat16, "w_q"), _ptr(s_q, torch.float32, "s_q"), _ptr(bias, torch.float32, "bias"),
+        _stream()), "stc_query_bias")
 
 
 def decode_attn(shape: Shape, cache: Cache, q: torch.Tensor, page_ids: Optional[torch.Tensor],

@@ -100,6 +100,9 @@ cudaError_t launch_append(const Geom& g, const void* k, void* kmin, void* kmax, 
 cudaError_t launch_router_logits(const Geom& g, const void* h, const void* w, const float* bias, int d_model,
                                  float* scores, int32_t* status, cudaStream_t st);
 
+cudaError_t launch_query_bias(int B, int Lq, int d_model, int n_logits, const void* h_q, const int32_t* q_len,
+                              const void* w_q, float* s_q, float* bias, cudaStream_t st);
+
 struct AttnPlan { int n_workers, slots_cap; };   // warps that share the pages; partial slots per problem
 AttnPlan attn_plan(const Geom& g, int max_pages);
 size_t attn_ws_bytes(const Geom& g, int max_pages);

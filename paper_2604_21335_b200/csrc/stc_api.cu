@@ -169,6 +169,18 @@ int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, 
                                         static_cast<cudaStream_t>(stream)));
 }
 
+int32_t stc_query_bias(int32_t batch, int32_t q_cap, int32_t d_model, int32_t n_logits, const void* h_q,
+                       const int32_t* q_len_opt, const void* w_q, float* s_q, float* bias, void* stream) {
+    if (batch < 0 || q_cap < 0 || d_model <= 0 || n_logits < 0 || batch > 65535) return STC_ERR_INVALID_ARG;
+    if (d_model % 8 != 0) return STC_ERR_UNSUPPORTED;
+    if (batch == 0) return STC_OK;
+    if (!s_q || (n_logits > 0 && (!w_q || !bias)) || (q_cap > 0 && !h_q)) return STC_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(h_q) | reinterpret_cast<uintptr_t>(w_q) | reinterpret_cast<uintptr_t>(s_q)) & 15u) != 0)
+        return STC_ERR_INVALID_ARG;
+    return cuda_rc(launch_query_bias(batch, q_cap, d_model, n_logits, h_q, q_len_opt, w_q, s_q, bias,
+                                     static_cast<cudaStream_t>(stream)));
+}
+
 int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const void* v,
                           const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
                           void* stream) {

@@ -20,6 +20,10 @@ def cpu_bits(t):
     return O.bf16_bits(t.cpu())
 
 
+def cpu_f32(t):
+    return t.detach().float().cpu().numpy()
+
+
 def gpu_pipeline(w, d, seq_len=None, budget=None, k_nominal=None, min_per_token=1, mode=Bd.MODE_GLOBAL,
                  tok_class="auto", cap_groups=None, q_index=0, want_scores=True, page_ids_override=None):
     """Full pass on the GPU: metadata, selection, routing+packing, attention.

@@ -53,3 +53,31 @@ def test_unsupported_shapes_are_refused_on_the_host():
     with pytest.raises(P.StcError) as e:
         P.router_logits(shape, x, w, sc, st)
     assert e.value.code == 2
+
+
+@pytest.mark.parametrize("B,Lq,dm,N", [
+    (1, 1, 64, 16),                     # one token: the mean is the row
+    (3, 37, 4096, 256),                 # LLaMA-2-7B router width, ragged region lengths
+    (2, 130, 264, 64),                  # d_model not a multiple of the 256-channel CTA slice
+])
+def test_query_summary_term_matches_the_checker_and_feeds_the_router(B, Lq, dm, N):
+    g = torch.Generator(device=DEV); g.manual_seed(B * 100 + Lq)
+    h_q = torch.randn(B, Lq, dm, generator=g, device=DEV).to(torch.bfloat16)
+    w_q = (torch.randn(N, dm, generator=g, device=DEV) / dm ** 0.5).to(torch.bfloat16)
+    q_len = torch.tensor([Lq, max(Lq // 3, 0), 0][:B], dtype=torch.int32, device=DEV)
+    s_q = torch.full((B, dm), float("nan"), dtype=torch.float32, device=DEV)
+    bias = torch.full((B, N), float("nan"), dtype=torch.float32, device=DEV)
+    P.query_bias(h_q, w_q, s_q, bias, q_len=q_len)
+    torch.cuda.synchronize()
+    s_o, b_o = O.query_bias(H.cpu_bits(h_q), H.cpu_bits(w_q), q_len.cpu().numpy())
+    # fp32 sums of n terms: worst case n * 2^-24 * sum|terms|; allow a tenth of it
+    mean_abs = np.stack([np.abs(H.cpu_f32(h_q)[b, : int(q_len[b])]).mean(axis=0) if int(q_len[b]) else np.zeros(dm)
+                         for b in range(B)])
+    tol_s = 0.1 * Lq * 2.0 ** -24 * mean_abs.max() + 1e-7
+    assert np.abs(s_q.double().cpu().numpy() - s_o).max() <= tol_s
+    tol_b = 0.1 * (dm + Lq) * 2.0 ** -24 * float((mean_abs @ np.abs(H.cpu_f32(w_q)).T).max()) + 1e-7
+    assert np.abs(bias.double().cpu().numpy() - b_o).max() <= tol_b
+    # a second call gives the same bits (fixed summation order)
+    s2, b2 = torch.empty_like(s_q), torch.empty_like(bias)
+    P.query_bias(h_q, w_q, s2, b2, q_len=q_len)
+    assert torch.equal(s2, s_q) and torch.equal(b2, bias)
