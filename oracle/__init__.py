@@ -112,10 +112,11 @@ def page_scores(q_group, kmin, kmax) -> np.ndarray:
     return u
 
 
-def select(u: np.ndarray, token_budget: int) -> np.ndarray:
+def select(u: np.ndarray, token_budget: int, n_recent_pages: int = 0) -> np.ndarray:
     u = np.ascontiguousarray(u, np.float32)
     ids = np.zeros(max(1, u.shape[0]), np.int32)
-    k = lib().stc_o_select(_p(u), C.c_int32(u.shape[0]), C.c_int32(token_budget), _p(ids))
+    k = lib().stc_o_select_recent(_p(u), C.c_int32(u.shape[0]), C.c_int32(token_budget),
+                                  C.c_int32(n_recent_pages), _p(ids))
     return ids[:k].copy()
 
 
@@ -186,7 +187,8 @@ def page_meta_batch(k, seq_len=None):
     return kmin, kmax
 
 
-def select_batch(q, kmin, kmax, token_budget, t_cap, seq_len=None, max_pages=None, want_scores=False):
+def select_batch(q, kmin, kmax, token_budget, t_cap, seq_len=None, max_pages=None, want_scores=False,
+                 n_recent_pages=0):
     """q uint16 [B,Hq,128] -> page_ids i32 [B,Hkv,max_pages], n_pages i32 [B,Hkv][, scores]."""
     B, Hq, _ = q.shape
     Hkv, P = kmin.shape[1], kmin.shape[2]
@@ -196,10 +198,10 @@ def select_batch(q, kmin, kmax, token_budget, t_cap, seq_len=None, max_pages=Non
     n = np.zeros((B, Hkv), np.int32)
     sc = np.zeros((B, Hkv, P), np.float32) if want_scores else None
     sl = None if seq_len is None else np.ascontiguousarray(seq_len, np.int32)
-    lib().stc_o_select_batch(C.c_int32(B), C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(t_cap), _p(sl),
-                             _p(np.ascontiguousarray(q), np.uint16), _p(np.ascontiguousarray(kmin), np.uint16),
-                             _p(np.ascontiguousarray(kmax), np.uint16), C.c_int32(token_budget),
-                             C.c_int32(max_pages), _p(ids), _p(n), _p(sc))
+    lib().stc_o_select_batch_recent(C.c_int32(B), C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(t_cap), _p(sl),
+                                    _p(np.ascontiguousarray(q), np.uint16), _p(np.ascontiguousarray(kmin), np.uint16),
+                                    _p(np.ascontiguousarray(kmax), np.uint16), C.c_int32(token_budget),
+                                    C.c_int32(n_recent_pages), C.c_int32(max_pages), _p(ids), _p(n), _p(sc))
     return (ids, n, sc) if want_scores else (ids, n)
 
 

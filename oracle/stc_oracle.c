@@ -161,6 +161,26 @@ int32_t stc_o_select(const float* u, int32_t n_pages, int32_t token_budget, int3
 }
 
 /* ------------------------------------------------------------------------
+ * Page selection with a local window (Appendix A, LLM training configuration:
+ * "Quest chunk/window size 16 / 64" -- read as Quest's always-attended window of
+ * the most recent tokens, here n_recent_pages whole pages, counted against the
+ * budget): with k_pg = min(n_pages, budget / 16) and w = min(n_recent_pages,
+ * k_pg), the last w pages are kept and the other k_pg - w are the best-scoring
+ * of the pages before them.  Ids ascending.  Returns k_pg.
+ * ---------------------------------------------------------------------- */
+int32_t stc_o_select_recent(const float* u, int32_t n_pages, int32_t token_budget,
+                            int32_t n_recent_pages, int32_t* page_ids) {
+    int32_t k_pg = token_budget / PAGE;
+    if (k_pg > n_pages) k_pg = n_pages;
+    if (k_pg < 0) k_pg = 0;
+    int32_t w = n_recent_pages < 0 ? 0 : n_recent_pages;
+    if (w > k_pg) w = k_pg;
+    int32_t kept = stc_o_select(u, n_pages - w, (k_pg - w) * PAGE, page_ids);
+    for (int32_t i = 0; i < w; ++i) page_ids[kept + i] = n_pages - w + i;
+    return kept + w;
+}
+
+/* ------------------------------------------------------------------------
  * Routing mask (Section 3.3 "Routing mask", Section 3.4 global budget,
  * Appendix B.1 M = N*K).
  *   scores [len][S]; cls [len] or NULL (all routed); mask [len] out.
@@ -388,10 +408,11 @@ void stc_o_page_meta_batch(int32_t B, int32_t Hkv, int32_t t_cap, const int32_t*
     }
 }
 
-void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
-                        const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax,
-                        int32_t token_budget, int32_t max_pages, int32_t* page_ids,
-                        int32_t* n_pages, float* scores_out /* [B][Hkv][p_cap] or NULL */) {
+void stc_o_select_batch_recent(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                               const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax,
+                               int32_t token_budget, int32_t n_recent_pages, int32_t max_pages,
+                               int32_t* page_ids, int32_t* n_pages,
+                               float* scores_out /* [B][Hkv][p_cap] or NULL */) {
     int32_t p_cap = (t_cap + PAGE - 1) / PAGE;
     int32_t gq = Hq / Hkv;
 #pragma omp parallel for schedule(static)
@@ -403,7 +424,7 @@ void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const
         int32_t* ids = (int32_t*)malloc(sizeof(int32_t) * (size_t)(p_cap + 1));
         stc_o_page_scores(q + ((size_t)b * Hq + (size_t)hk * gq) * D, gq,
                           kmin + (size_t)pr * p_cap * D, kmax + (size_t)pr * p_cap * D, np, u);
-        int32_t kp = stc_o_select(u, np, token_budget, ids);
+        int32_t kp = stc_o_select_recent(u, np, token_budget, n_recent_pages, ids);
         if (kp > max_pages) kp = max_pages;   /* caller sized the list too small: truncated */
         memcpy(page_ids + (size_t)pr * max_pages, ids, sizeof(int32_t) * (size_t)kp);
         n_pages[pr] = kp;
@@ -411,6 +432,14 @@ void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const
         free(u);
         free(ids);
     }
+}
+
+void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                        const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax,
+                        int32_t token_budget, int32_t max_pages, int32_t* page_ids,
+                        int32_t* n_pages, float* scores_out) {
+    stc_o_select_batch_recent(B, Hq, Hkv, t_cap, seq_len, q, kmin, kmax, token_budget, 0, max_pages, page_ids,
+                              n_pages, scores_out);
 }
 
 /* status [B*Hkv]: 0 ok, -1 budget below one group per token, -2 bad args,

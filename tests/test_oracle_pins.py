@@ -489,3 +489,22 @@ def test_query_bias_is_the_mean_of_the_per_token_logits():
         want = per_tok[b, :, : q_len[b], :].mean(axis=1).reshape(-1)
         np.testing.assert_allclose(bias[b], want, rtol=0, atol=1e-12)
         np.testing.assert_allclose(s_q[b], f32(hq)[b, : q_len[b]].astype(np.float64).mean(axis=0), rtol=0, atol=1e-14)
+
+
+# ---------------------------------------------------------------------- selection with a recent window
+def test_select_recent_window_against_brute_force():
+    g = np.random.default_rng(31)
+    for n, budget, w in [(40, 160, 4), (40, 160, 0), (40, 160, 10), (40, 160, 25), (7, 1000, 3), (33, 16, 4),
+                         (50, 320, 20), (12, 0, 2)]:
+        u = g.integers(0, 6, n).astype(np.float32)            # many ties
+        ids = O.select(u, budget, w)
+        k = min(n, budget // 16)
+        ww = min(w, k)
+        window = list(range(n - ww, n))
+        # exhaustive: rank the pages before the window by (-score, id), take k - ww of them
+        rest = sorted(range(n - ww), key=lambda p: (-u[p], p))[: k - ww]
+        assert ids.tolist() == sorted(rest + window), (n, budget, w)
+        assert len(set(ids.tolist())) == k
+    # no window = the plain rule
+    u = g.standard_normal(64).astype(np.float32)
+    np.testing.assert_array_equal(O.select(u, 256, 0), O.select(u, 256))
