@@ -128,6 +128,18 @@ int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const v
                          int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
                          void* stream);
 
+/* stc_quest_select with Quest's local window (Appendix A, LLM training
+ * configuration: "Quest chunk/window size 16 / 64", i.e. a window of 64 recent
+ * tokens = 4 pages next to 16-token chunks): with w = min(n_recent_pages,
+ * k_pg), the last w valid pages of every problem are always kept and count
+ * against the budget; the other k_pg - w pages are the best-scoring of the
+ * pages before them (same bound, same tie rule, ids ascending).
+ * n_recent_pages = 0 is stc_quest_select.  Same arguments otherwise. */
+int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, const void* q,
+                                int32_t token_budget, int32_t n_recent_pages, int32_t max_pages,
+                                int32_t* page_ids, int32_t* n_pages, float* scores_opt, void* ws,
+                                size_t ws_bytes, void* stream);
+
 /* stc_quest_select for callers that cannot provide a workspace.  (The paper has
  * no counterpart: this is a deployment convenience of the library.)
  *

@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window",
 )
 
 
@@ -70,6 +70,9 @@ def load_library():
         lib.stc_build_page_meta.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_int32, C.c_int32, C.c_void_p]
         lib.stc_quest_select.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32, C.c_int32,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.stc_quest_select_window.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32, C.c_int32,
+                                                C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                                C.c_void_p]
         lib.stc_quest_select_static.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32,
                                                 C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_route_pack.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
@@ -193,8 +196,17 @@ def build_page_meta(shape: Shape, cache: Cache, page_begin: int = 0, page_end: i
 
 
 def quest_select(shape: Shape, cache: Cache, q: torch.Tensor, token_budget: int, page_ids: torch.Tensor,
-                 n_pages: torch.Tensor, ws: torch.Tensor, scores: Optional[torch.Tensor] = None) -> None:
+                 n_pages: torch.Tensor, ws: torch.Tensor, scores: Optional[torch.Tensor] = None,
+                 n_recent_pages: int = 0) -> None:
+    """n_recent_pages > 0 keeps that many most recent pages unconditionally (stc_quest_select_window)."""
     cs, cc = shape.c(), cache.c()
+    if n_recent_pages:
+        _check(load_library().stc_quest_select_window(
+            C.byref(cs), C.byref(cc), _ptr(q, torch.bfloat16, "q"), token_budget, n_recent_pages,
+            page_ids.shape[-1], _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"),
+            _ptr(scores, torch.float32, "scores"), _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()),
+            "stc_quest_select_window")
+        return
     _check(load_library().stc_quest_select(
         C.byref(cs), C.byref(cc), _ptr(q, torch.bfloat16, "q"), token_budget, page_ids.shape[-1],
         _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"),

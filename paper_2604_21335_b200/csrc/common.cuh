@@ -81,7 +81,7 @@ cudaError_t launch_page_meta(const Geom& g, const void* k, void* kmin, void* kma
 
 size_t select_ws_bytes(const Geom& g);
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
-                                int token_budget, int max_pages, int32_t* page_ids,
+                                int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
                                 int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st);
 
 size_t route_ws_bytes(const Geom& g);

@@ -302,7 +302,7 @@ template <int GQ>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ kmax,
                     const uint4* __restrict__ q, const int32_t* __restrict__ seq_len, int Hq, int Hkv,
-                    int T, int P, int token_budget, int max_pages, int32_t* __restrict__ page_ids,
+                    int T, int P, int token_budget, int n_recent, int max_pages, int32_t* __restrict__ page_ids,
                     int32_t* __restrict__ n_pages, float* __restrict__ scores, int scores_wanted,
                     unsigned* __restrict__ counters, int units_per_problem, long long total_units) {
     constexpr bool kSplit = GQ > 4;            // halves of a warp share a page, split the heads
@@ -429,7 +429,10 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             __threadfence();
             int32_t* ids = page_ids + (size_t)problem * max_pages;
             // the copy ring is idle here (all copies have landed): it stages the keys
-            block_topk(scores + row0, np, k_pg, ids, ring_mem, s_topk);
+            // the local window: the last w pages are kept, the rest of the budget goes to the pages before them
+            const int w = min(max(n_recent, 0), k_pg);
+            if (k_pg > w) block_topk(scores + row0, np - w, k_pg - w, ids, ring_mem, s_topk);
+            for (int i = tid; i < w; i += kThreads) ids[k_pg - w + i] = np - w + i;
             if (tid == 0) n_pages[problem] = k_pg;
         }
     }
@@ -455,7 +458,7 @@ size_t select_ws_bytes(const Geom& g) {
 }
 
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
-                                int token_budget, int max_pages, int32_t* page_ids,
+                                int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
                                 int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st) {
     if (g.problems == 0) return cudaSuccess;
     unsigned* counters = static_cast<unsigned*>(ws);
@@ -475,7 +478,7 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
         quest_select_kernel<GQ_><<<(unsigned)grid, kThreads, kRingBytes, st>>>(                      \
             static_cast<const uint4*>(kmin), static_cast<const uint4*>(kmax),                        \
             static_cast<const uint4*>(q), g.seq_len, g.Hq, g.Hkv, g.T, g.P, token_budget,            \
-            max_pages, page_ids, n_pages, scores, scores_opt != nullptr, counters,                   \
+            n_recent_pages, max_pages, page_ids, n_pages, scores, scores_opt != nullptr, counters,                   \
             units_per_problem, total_units);                                                         \
         break;
     switch (g.Gq) {

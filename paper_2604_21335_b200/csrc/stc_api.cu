@@ -88,17 +88,25 @@ int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const v
                          int32_t token_budget, int32_t max_pages, int32_t* page_ids,
                          int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
                          void* stream) {
+    return stc_quest_select_window(shape, cache, q, token_budget, 0, max_pages, page_ids, n_pages, scores_opt, ws,
+                                   ws_bytes, stream);
+}
+
+int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, const void* q,
+                                int32_t token_budget, int32_t n_recent_pages, int32_t max_pages,
+                                int32_t* page_ids, int32_t* n_pages, float* scores_opt, void* ws,
+                                size_t ws_bytes, void* stream) {
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
-    if (!cache || token_budget < 0 || max_pages < 0) return STC_ERR_INVALID_ARG;
+    if (!cache || token_budget < 0 || max_pages < 0 || n_recent_pages < 0) return STC_ERR_INVALID_ARG;
     if (empty(g)) return STC_OK;
     if (!cache->kmin || !cache->kmax || !q || !page_ids || !n_pages) return STC_ERR_INVALID_ARG;
     const int want = token_budget / kPage < g.P ? token_budget / kPage : g.P;
     if (max_pages < want) return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, select_ws_bytes(g));
     if (rc != STC_OK) return rc;
-    return cuda_rc(launch_quest_select(g, cache->kmin, cache->kmax, q, token_budget, max_pages,
+    return cuda_rc(launch_quest_select(g, cache->kmin, cache->kmax, q, token_budget, n_recent_pages, max_pages,
                                        page_ids, n_pages, scores_opt, ws,
                                        static_cast<cudaStream_t>(stream)));
 }
