@@ -277,3 +277,24 @@ def test_full_size_sampled_problems(name, samples):
         H.assert_bit_exact_write_side(w1, g1, o)
         H.assert_bit_exact_selection(g1, o)
         H.assert_attention_close(g1, o)
+
+
+@pytest.mark.parametrize("name,S,T", [("cfg0", 8, 1300), ("cfg2", 16, 16 * 70 + 3)])
+def test_many_medium_problems_span_the_ranges_of_the_selection_ctas(name, S, T):
+    """Hundreds of problems, each a few 256-token units long (too long for the one-CTA kernel):
+    the persistent selection kernel's CTAs then own ranges that cross problem boundaries, and
+    several CTAs share a problem.  Ragged lengths, a class mix and an empty sequence."""
+    w0 = W.get(name)
+    w = W.shrink(w0, batch=40, n_q_heads=8 * w0.gq, n_kv_heads=8, t_cache=T, token_budget=16 * 20)
+    d = W.make_inputs(w, DEV)
+    g0 = torch.Generator(device="cpu"); g0.manual_seed(77)
+    seq = torch.randint(1, T + 1, (40,), generator=g0, dtype=torch.int32)
+    seq[3] = 0; seq[7] = T; seq[11] = 257
+    cls = torch.randint(0, 3, (40, T), generator=g0, dtype=torch.uint8)
+    cls[5] = 1; cls[6] = 2
+    seq_d, cls_d = seq.to(DEV), cls.to(DEV)
+    g = H.gpu_pipeline(w, d, seq_len=seq_d, tok_class=cls_d)
+    o = H.oracle_pipeline(w, d, seq_len=seq.numpy(), tok_class=cls)
+    H.assert_bit_exact_write_side(w, g, o)
+    H.assert_bit_exact_selection(g, o)
+    H.assert_attention_close(g, o)
