@@ -624,6 +624,8 @@ AttnPlan attn_plan(const Geom& g, int max_pages) {
     if (workers > wave) workers = wave;
     // a call that fits one CTA per SM runs there, with the deeper ring
     if (workers > 148LL * kWarps && workers < 148LL * kWarps * 3 / 2) workers = 148LL * kWarps;
+    // many short problems: one warp per problem, so that no problem is split and nothing is merged
+    if (g.problems <= wave && 2LL * g.problems >= workers) workers = g.problems;
     const long long by_slots = (long long)(kMaxSlots - 1) * (g.problems < 1 ? 1 : g.problems);
     if (workers > by_slots) workers = by_slots;  // keeps ceil(workers / problems) + 1 <= kMaxSlots
     if (workers < 1) workers = 1;
