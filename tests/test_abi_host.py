@@ -78,6 +78,16 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, None, fake, 16, st) == 3
     assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, None, 64, 0.1, fake, None, fake, 1 << 30, st) == 1
     assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, fake, 64, 0.1, fake, None, fake, 16, st) == 3
+    # the window variant: a negative window is an argument error, a valid one reaches the workspace check
+    assert lib.stc_quest_select_window(C.byref(cs), C.byref(cc), fake, 1024, -1, 64, fake, fake, None, fake, 1 << 30, st) == 1
+    assert lib.stc_quest_select_window(C.byref(cs), C.byref(cc), fake, 1024, 4, 64, fake, fake, None, None, 0, st) == 3
+    # query summary: sizes, alignment and the multiple-of-8 rule are checked on the host
+    assert lib.stc_query_bias(-1, 4, 64, 16, fake, None, fake, fake, fake, st) == 1
+    assert lib.stc_query_bias(2, 4, 0, 16, fake, None, fake, fake, fake, st) == 1
+    assert lib.stc_query_bias(2, 4, 60, 16, fake, None, fake, fake, fake, st) == 2
+    assert lib.stc_query_bias(2, 4, 64, 16, C.c_void_p(0x1008), None, fake, fake, fake, st) == 1
+    assert lib.stc_query_bias(2, 4, 64, 16, fake, None, fake, None, fake, st) == 1
+    assert lib.stc_query_bias(0, 4, 64, 16, None, None, None, None, None, st) == 0
 
 
 def test_cache_bytes_reproduces_the_closed_form(lib):
