@@ -400,10 +400,13 @@ def run_gpu(args, r: D.Rank):
     read_ms = per_call_ms[3] + per_call_ms[4]
     read_bytes = ab["quest_select"] + ab["decode_attn"]
     read_gbs = read_bytes / (read_ms * 1e-3) / 1e9
-    # dominant single-kernel call of the step (route_mask is a chain of four kernels)
-    single = {n: per_call_ms[c] for c, n in enumerate(names) if ab[n] and n != "route_mask"}
+    # dominant call of the step (every call is one kernel)
+    single = {n: per_call_ms[c] for c, n in enumerate(names) if ab[n]}
     dom = max(single, key=single.get)
-    roof = {"bound": "hbm", "kernel": KERNEL_OF[dom], "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
+    kernel_of = dict(KERNEL_OF)
+    if (T + 255) // 256 <= 32 // S:                      # problems that fit one CTA take the small selection kernel
+        kernel_of["route_mask"] = "route_select_small_kernel"
+    roof = {"bound": "hbm", "kernel": kernel_of[dom], "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
             "frac": round(per_kernel[dom]["GBps"] / peak, 4), "peak_source": peak_src + " copy bandwidth",
             "traffic": TRAFFIC_NOTE.get((args.workload, dom))}
     line = {

@@ -205,7 +205,7 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
  * values are available (or want to time them apart).  stc_route_mask is the
  * routing-mask rule of stc_route_pack (same passages, same arguments): it
  * leaves in out->v_mask the groups every token keeps for certain and, in the
- * workspace, the groups tied at the selection threshold and the per-tile
+ * workspace, the groups tied at the selection threshold and the per-unit
  * counts.  stc_pack_values turns that into the final masks (ties resolved to
  * the lowest flat indices), the offsets, the packed store, totals and status.
  * It must be the next use of the same workspace after stc_route_mask, with
