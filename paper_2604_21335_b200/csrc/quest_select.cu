@@ -298,21 +298,16 @@ __device__ __forceinline__ float reduce_heads(float (&v)[NH], int l, unsigned hm
     return x;
 }
 
-// Three or more query heads per KV head: the two halves of a warp share a page and split the
-// heads (two per lane up to four heads, four per lane up to eight), which halves the query
-// registers of a lane; up to four heads that makes room for a third CTA per SM.
-__host__ __device__ constexpr int ctas_per_sm(int gq) { return (gq == 3 || gq == 4) ? 3 : kCtasPerSm; }
-
 template <int GQ>
-__global__ void __launch_bounds__(kThreads, ctas_per_sm(GQ))
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ kmax,
                     const uint4* __restrict__ q, const int32_t* __restrict__ seq_len, int Hq, int Hkv,
                     int T, int P, int token_budget, int n_recent, int max_pages, int32_t* __restrict__ page_ids,
                     int32_t* __restrict__ n_pages, float* __restrict__ scores, int scores_wanted,
                     unsigned* __restrict__ counters, int units_per_problem, long long total_units) {
-    constexpr bool kSplit = GQ > 2;            // halves of a warp share a page, split the heads
-    constexpr int NH = kSplit ? (GQ > 4 ? 4 : 2) : GQ;    // heads per lane: 1 / 2 / 4
-    constexpr int kPagesPerUnit = kWarps * 2;  // a warp owns two pages of a unit (one per half, or both in turn)
+    constexpr bool kSplit = GQ > 4;            // halves of a warp share a page, split the heads
+    constexpr int NH = kSplit ? 4 : (GQ == 3 ? 4 : GQ);   // heads per lane, padded to 1 / 2 / 4
+    constexpr int kPagesPerUnit = kWarps * (kSplit ? 1 : 2);
 
     extern __shared__ __align__(16) uint32_t ring_mem[];
     __shared__ uint32_t s_topk[kTopkSmemWords];
@@ -320,16 +315,13 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int half = lane >> 4, l = lane & 15;
-    const int sub = kSplit ? warp * 2 : warp * 2 + half;   // this half-warp's (first) page inside a unit
+    const int sub = kSplit ? warp : warp * 2 + half;       // this half-warp's page inside a unit
     const unsigned hm = kSplit ? 0xFFFFFFFFu : (0xFFFFu << (16 * half));
     const long long x1 = total_units * (blockIdx.x + 1) / gridDim.x;
     long long x = total_units * blockIdx.x / gridDim.x;
 
-    // ring slot, per warp 1 KiB.  Unsplit: 512 B of kmin chunks (two pages) then 512 B of kmax chunks,
-    // every lane copies and reads its own two chunks.  Split: page A = 256 B kmin (copied by lanes
-    // 0-15) + 256 B kmax (lanes 16-31), then page B the same; every lane reads chunk l of all four.
+    // ring slot: per warp 512 B of kmin chunks then 512 B of kmax chunks (conflict-free)
     const uint32_t ring = smem_u32(ring_mem) + (uint32_t)warp * 1024u + (uint32_t)lane * 16u;
-    const uint32_t ring_rd = smem_u32(ring_mem) + (uint32_t)warp * 1024u + (uint32_t)l * 16u;
     constexpr uint32_t kSlotBytes = kThreads * 32u;
 
 #pragma unroll 1
@@ -353,19 +345,15 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
 
         const size_t row0 = (size_t)problem * P;
         // units of the segment in which this half-warp's page exists (pages advance by
-        // kPagesPerUnit per unit, so validity is a prefix of the units); split: pages A and B = A + 1
+        // kPagesPerUnit per unit, so validity is a prefix of the units)
         const int page0 = u_begin * kPagesPerUnit + sub;
         const int lim = max(0, min(n, (np - page0 + kPagesPerUnit - 1) / kPagesPerUnit));
-        const int lim_b = kSplit ? max(0, min(n, (np - page0 - 1 + kPagesPerUnit - 1) / kPagesPerUnit)) : 0;
         // running source pointers / ring slot of the next unit to issue (units are issued in order)
-        const uint4* src_min = (kSplit && half ? kmax : kmin) + (row0 + page0) * kOctets + l;   // split: the lane's one source
+        const uint4* src_min = kmin + (row0 + page0) * kOctets + l;
         const uint4* src_max = kmax + (row0 + page0) * kOctets + l;
         uint32_t slot_off = 0;
         auto issue = [&](int i) {                 // unit i of the segment -> slot i % kDepth
-            if (kSplit) {
-                if (i < lim) cp_async16(ring + slot_off, src_min);
-                if (i < lim_b) cp_async16(ring + slot_off + 512u, src_min + kOctets);
-            } else if (i < lim) {
+            if (i < lim) {
                 cp_async16(ring + slot_off, src_min);
                 cp_async16(ring + slot_off + 512u, src_max);
             }
@@ -382,7 +370,7 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
         uint64_t qp2[NH][4], qn2[NH][4];           // (even, odd) channel pairs of q+ and q-
 #pragma unroll
         for (int h = 0; h < NH; ++h) {
-            const int head = min(kSplit ? half * NH + h : h, GQ - 1);   // padding repeats a real head
+            const int head = min(kSplit ? half * 4 + h : h, GQ - 1);   // padding repeats a real head
             const uint4 qw = q[((size_t)b * Hq + (size_t)hk * GQ + head) * kOctets + l];
             const uint32_t w[4] = {qw.x, qw.y, qw.z, qw.w};
 #pragma unroll
@@ -392,7 +380,7 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                 qn2[h][i] = pack2(fminf(e, 0.f), fminf(o, 0.f));
             }
         }
-        auto score_page = [&](const uint4& lo, const uint4& hi) -> float {
+        auto score_unit = [&](int i, const uint4& lo, const uint4& hi) {
             const uint32_t wl[4] = {lo.x, lo.y, lo.z, lo.w}, wh[4] = {hi.x, hi.y, hi.z, hi.w};
             uint64_t a2[4], z2[4];
 #pragma unroll
@@ -410,41 +398,21 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             }
             float best = reduce_heads<NH>(v, l, hm);
             if (kSplit) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, 16));
-            return best;
+            if (writer && i < lim) *dst_score = best;
+            dst_score += kPagesPerUnit;
         };
 
 #pragma unroll 1
         for (int i = 0; i < n; i += 2) {
             cp_async_wait<kDepth - 2>();           // units i and i+1 have landed
-            const uint32_t o0 = (uint32_t)(i & (kDepth - 1)) * kSlotBytes;
-            const uint32_t o1 = (uint32_t)((i + 1) & (kDepth - 1)) * kSlotBytes;
-            if (kSplit) {
-                __syncwarp();                      // the other half's copies are complete, too
-                const uint4 la0 = lds16(ring_rd + o0), ha0 = lds16(ring_rd + o0 + 256u);
-                const uint4 lb0 = lds16(ring_rd + o0 + 512u), hb0 = lds16(ring_rd + o0 + 768u);
-                const float a0 = score_page(la0, ha0), b0 = score_page(lb0, hb0);
-                const uint4 la1 = lds16(ring_rd + o1), ha1 = lds16(ring_rd + o1 + 256u);
-                const uint4 lb1 = lds16(ring_rd + o1 + 512u), hb1 = lds16(ring_rd + o1 + 768u);
-                __syncwarp();                      // every lane has read both slots: they may be refilled
-                issue(i + kDepth);
-                issue(i + kDepth + 1);
-                const float a1 = score_page(la1, ha1), b1 = score_page(lb1, hb1);
-                if (writer) {
-                    if (i < lim) dst_score[0] = a0;
-                    if (i < lim_b) dst_score[1] = b0;
-                    if (i + 1 < lim) dst_score[kPagesPerUnit] = a1;
-                    if (i + 1 < lim_b) dst_score[kPagesPerUnit + 1] = b1;
-                }
-            } else {
-                const uint4 lo0 = lds16(ring + o0), hi0 = lds16(ring + o0 + 512u);
-                const uint4 lo1 = lds16(ring + o1), hi1 = lds16(ring + o1 + 512u);
-                const float s0 = score_page(lo0, hi0), s1 = score_page(lo1, hi1);
-                if (writer && i < lim) dst_score[0] = s0;
-                if (writer && i + 1 < lim) dst_score[kPagesPerUnit] = s1;
-                issue(i + kDepth);                 // refill the two slots just read
-                issue(i + kDepth + 1);
-            }
-            dst_score += 2 * kPagesPerUnit;
+            const uint32_t s0 = ring + (uint32_t)(i & (kDepth - 1)) * kSlotBytes;
+            const uint32_t s1 = ring + (uint32_t)((i + 1) & (kDepth - 1)) * kSlotBytes;
+            const uint4 lo0 = lds16(s0), hi0 = lds16(s0 + 512u);
+            const uint4 lo1 = lds16(s1), hi1 = lds16(s1 + 512u);
+            score_unit(i, lo0, hi0);
+            score_unit(i + 1, lo1, hi1);
+            issue(i + kDepth);                     // refill the two slots just read
+            issue(i + kDepth + 1);
         }
         cp_async_wait<0>();
         if (trivial) continue;
@@ -498,10 +466,10 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
                                : reinterpret_cast<float*>(static_cast<char*>(ws) + counters_bytes(g));
     cudaError_t e = cudaMemsetAsync(counters, 0, (size_t)g.problems * 4, st);
     if (e != cudaSuccess) return e;
-    const int pages_per_unit = kWarps * 2;
+    const int pages_per_unit = kWarps * (g.Gq > 4 ? 1 : 2);
     const int units_per_problem = (g.P + pages_per_unit - 1) / pages_per_unit;
     const long long total_units = (long long)units_per_problem * g.problems;
-    long long grid = (long long)sm_count() * ctas_per_sm(g.Gq);
+    long long grid = (long long)sm_count() * kCtasPerSm;
     if (grid > total_units) grid = total_units;
 #define STC_SEL(GQ_)                                                                                 \
     case GQ_:                                                                                        \
