@@ -298,3 +298,69 @@ def test_many_medium_problems_span_the_ranges_of_the_selection_ctas(name, S, T):
     H.assert_bit_exact_write_side(w, g, o)
     H.assert_bit_exact_selection(g, o)
     H.assert_attention_close(g, o)
+
+
+def test_benchmark_launch_configuration_full_size():
+    """cfg1 at full size, launched the way the benchmark times it: the key side (metadata, page
+    selection) and the value side (routing masks, packing) on two streams inside one CUDA graph,
+    joined before the attention call, replayed several times with rotating queries; sampled
+    problems of the last replay against the checker."""
+    w = W.get("cfg1")
+    NQ = 3
+    d = W.make_inputs(w, DEV, n_queries=NQ)
+    B, Hkv, Hq, T, S = w.batch, w.n_kv_heads, w.n_q_heads, w.t_cache, w.n_groups
+    shape = P.Shape(B, Hq, Hkv, S, T, d["seq_len"])
+    cache = P.Cache.allocate(shape, d["k"], T * w.k_nominal)
+    total = torch.zeros(B, Hkv, dtype=torch.int64, device=DEV)
+    status = torch.full((B, Hkv), -1, dtype=torch.int32, device=DEV)
+    max_pages = w.token_budget // 16
+    ids = torch.full((B, Hkv, max_pages), -1, dtype=torch.int32, device=DEV)
+    npg = torch.full((B, Hkv), -1, dtype=torch.int32, device=DEV)
+    u = torch.full((B, Hkv, shape.n_pages), float("nan"), dtype=torch.float32, device=DEV)
+    out = torch.full((B, Hq, 128), float("nan"), dtype=torch.float32, device=DEV)
+    lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device=DEV)
+    ws_r = Bd.new_workspace(shape, Bd.OP_ROUTE_PACK, device=DEV)
+    ws_s = Bd.new_workspace(shape, Bd.OP_QUEST_SELECT, device=DEV)
+    ws_a = Bd.new_workspace(shape, Bd.OP_DECODE_ATTN, max_pages, device=DEV)
+    qs = [d["q"][i].contiguous() for i in range(NQ)]
+    side = torch.cuda.Stream()
+
+    def step(i):
+        main = torch.cuda.current_stream()
+        side.wait_stream(main)
+        with torch.cuda.stream(side):
+            P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)
+            P.pack_values(shape, d["v"], cache, total, status, ws_r)
+        P.build_page_meta(shape, cache)
+        P.quest_select(shape, cache, qs[i], w.token_budget, ids, npg, ws_s, scores=u)
+        main.wait_stream(side)
+        P.decode_attn(shape, cache, qs[i], ids, npg, H.SM_SCALE, out, ws_a, lse=lse)
+
+    step(0)
+    torch.cuda.synchronize()
+    graphs = []
+    for i in range(NQ):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step(i)
+        graphs.append(g)
+    for rep in range(3):
+        for g in graphs:
+            g.replay()
+    torch.cuda.synchronize()
+    assert (status == 0).all() and int(ws_a[:4].view(torch.int32)[0]) == 0
+    last = NQ - 1
+    for b, hk in [(0, 5), (0, 30)]:
+        w1, d1 = _problem_slice(w, d, b, hk)
+        o = H.oracle_pipeline(w1, d1, q_index=last)
+        g1 = dict(cache=P.Cache(kmin=cache.kmin[b:b + 1, hk:hk + 1].contiguous(),
+                                kmax=cache.kmax[b:b + 1, hk:hk + 1].contiguous(),
+                                v_mask=cache.v_mask[b:b + 1, hk:hk + 1].contiguous(),
+                                v_offs=cache.v_offs[b:b + 1, hk:hk + 1].contiguous(),
+                                v_packed=cache.v_packed[b:b + 1, hk:hk + 1].contiguous()),
+                  total=total[b:b + 1, hk:hk + 1], status=status[b:b + 1, hk:hk + 1],
+                  page_ids=ids[b:b + 1, hk:hk + 1], n_pages=npg[b:b + 1, hk:hk + 1], u=u[b:b + 1, hk:hk + 1],
+                  out=out[b:b + 1, hk * w.gq:(hk + 1) * w.gq], lse=lse[b:b + 1, hk * w.gq:(hk + 1) * w.gq])
+        H.assert_bit_exact_write_side(w1, g1, o)
+        H.assert_bit_exact_selection(g1, o)
+        H.assert_attention_close(g1, o)
