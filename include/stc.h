@@ -96,7 +96,7 @@ int32_t stc_version(void);
  * calls that share a workspace must not overlap on the device. */
 int32_t stc_workspace_bytes(const stc_shape* shape, int32_t op, int64_t arg, size_t* bytes_host);
 
-/* Page metadata (Quest chunk size 16: Appendix B.1, "LLM training
+/* Page metadata (Quest chunk size 16: Appendix C.1, table "LLM training
  * configuration"): for pages page_begin <= p < page_end (page_end < 0 = all)
  * and every channel c,
  *     kmin[p][c] = min_t k[t][c],  kmax[p][c] = max_t k[t][c]
@@ -128,9 +128,9 @@ int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const v
                          int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
                          void* stream);
 
-/* stc_quest_select with Quest's local window (Appendix A, LLM training
- * configuration: "Quest chunk/window size 16 / 64", i.e. a window of 64 recent
- * tokens = 4 pages next to 16-token chunks): with w = min(n_recent_pages,
+/* stc_quest_select with Quest's local window (Appendix C.1, table "LLM training
+ * configuration", which lists a Quest window of 64 next to the chunk of 16: read
+ * as a window of the 64 most recent tokens = 4 pages): with w = min(n_recent_pages,
  * k_pg), the last w valid pages of every problem are always kept and count
  * against the budget; the other k_pg - w pages are the best-scoring of the
  * pages before them (same bound, same tie rule, ids ascending).
@@ -217,7 +217,7 @@ int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_
 int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
                         int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream);
 
-/* Value-group router logits (Appendix A.1 "Value-Group Router": one linear
+/* Value-group router logits (Appendix B.1 "Value-Group Router": one linear
  * projection from the layer's input hidden state to S group logits per KV
  * head; Section 3.4's query-aware form g(h, s_Q) is the same projection with an
  * additive per-sequence term, passed as bias_opt):
@@ -252,8 +252,8 @@ int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, 
 int32_t stc_query_bias(int32_t batch, int32_t q_cap, int32_t d_model, int32_t n_logits, const void* h_q,
                        const int32_t* q_len_opt, const void* w_q, float* s_q, float* bias, void* stream);
 
-/* Streaming append (Section 3.4: "query-region tokens are not compressed" -- the
- * tokens generated during decoding keep their full values).  For every sequence
+/* Streaming append (Section 3.4 exempts the query region from value compression:
+ * the tokens generated during decoding keep all their value groups).  For every sequence
  * b the tokens old_len[b] <= t < len[b] (len = shape->seq_len AFTER the append,
  * or t_cap when seq_len is NULL) have just been added: their keys are already in
  * cache->k and their values in v (same [B][Hkv][T][128] layout as stc_route_pack;
@@ -297,7 +297,7 @@ int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const vo
                         void* stream);
 
 /* Stored bytes of the compressed cache for the accounting of Section 3.3
- * ("Compression ratio") and Appendix B.2: full-width keys of the retained
+ * ("Compression ratio") and Appendix C.2 ("SubToken configuration and budget"): full-width keys of the retained
  * tokens plus the packed groups (mask/offset/metadata bytes are returned
  * separately).  Host arithmetic only. */
 int32_t stc_cache_bytes(int64_t n_tokens_retained, int64_t n_groups_kept, int32_t n_groups,

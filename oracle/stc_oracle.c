@@ -47,7 +47,7 @@ static int32_t bf16_order(uint16_t b) {
 
 /* ------------------------------------------------------------------------
  * Page metadata: per page and channel, the minimum and maximum key over the
- * page's valid tokens.  (Quest chunk size 16: Appendix B.1, Table "LLM
+ * page's valid tokens.  (Quest chunk size 16: Appendix C.1, Table "LLM
  * training configuration"; the page statistic is Quest's per-channel bound.)
  * k [len..][128], kmin/kmax [ceil(len/16)][128].
  * ---------------------------------------------------------------------- */
@@ -161,9 +161,9 @@ int32_t stc_o_select(const float* u, int32_t n_pages, int32_t token_budget, int3
 }
 
 /* ------------------------------------------------------------------------
- * Page selection with a local window (Appendix A, LLM training configuration:
- * "Quest chunk/window size 16 / 64" -- read as Quest's always-attended window of
- * the most recent tokens, here n_recent_pages whole pages, counted against the
+ * Page selection with a local window (Appendix C.1, LLM training configuration:
+ * the table lists a Quest window of 64 beside the chunk of 16 -- read as Quest's
+ * always-attended window of the most recent tokens, here n_recent_pages whole pages, counted against the
  * budget): with k_pg = min(n_pages, budget / 16) and w = min(n_recent_pages,
  * k_pg), the last w pages are kept and the other k_pg - w are the best-scoring
  * of the pages before them.  Ids ascending.  Returns k_pg.
@@ -366,7 +366,7 @@ void stc_o_attend_masked_dense(const uint16_t* q, const uint16_t* k, const uint1
 }
 
 /* Retained-KV fraction by counting stored bytes (Section 3.3 "Compression
- * ratio", Appendix B.2: rho_total = r * (1 + K/S) / 2): full-width keys of the
+ * ratio", Appendix C.2: rho_total = r * (1 + K/S) / 2): full-width keys of the
  * retained tokens plus the packed value groups, over dense keys + values of
  * all original tokens. */
 double stc_o_kv_fraction(int64_t n_tokens_original, int64_t n_tokens_retained,
@@ -504,7 +504,7 @@ void stc_o_attend_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const
 }
 
 /* ------------------------------------------------------------------------
- * Value-group router (Appendix A.1 "Value-Group Router": a single linear
+ * Value-group router (Appendix B.1 "Value-Group Router": a single linear
  * projection from the layer input hidden state to S group logits; Section 3.4
  * gives the LLM form a = g(h, s_Q), read here as the same linear map applied to
  * [h ; s_Q], whose s_Q part is one additive vector per sequence).

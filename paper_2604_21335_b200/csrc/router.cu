@@ -1,6 +1,6 @@
 // Value-group router logits: scores[b][hk][t][j] = sum_c h[b][t][c] * w[hk*S+j][c] (+ bias).
 //
-// This is the one dense contraction of the method (Appendix A.1: the router is a
+// This is the one dense contraction of the method (Appendix B.1: the router is a
 // single linear projection of the layer's hidden state to S group logits), so it
 // runs on the 5th-generation tensor cores: a [tokens x d_model] . [d_model x Hkv*S]
 // GEMM with both operands K-major, bf16 in, fp32 accumulate.

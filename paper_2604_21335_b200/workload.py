@@ -8,7 +8,7 @@ Shapes follow the paper's settings: LLaMA-2-7B-like multi-head attention,
 Qwen2.5-7B-like grouped-query attention, a LLaVA-1.5-7B-like cache of 576
 visual + text tokens reduced to a quarter of the visual tokens (Appendix
 "Training Details and Implementation Cost", VLM paragraph), value groups
-S in {8, 16} with K/S budgets from Section 3.3 / Appendix B.
+S in {8, 16} with K/S budgets from Section 3.3 / Appendix C.
 
 Value recipe (all configs): Q, K, V iid N(0,1) rounded to bf16; in K, four
 channels per KV head (ids drawn once per head from the seed) are multiplied

@@ -1,6 +1,6 @@
 """Streaming append (stc_append_tokens): a decode loop that grows the cache one token at a
 time must end in exactly the state the CPU checker reaches when it routes the original
-tokens and keeps the appended ones at full width (query-region tokens are not compressed),
+tokens and keeps the appended ones at full width (Section 3.4 leaves the query region uncompressed),
 and attention over that state must agree with the checker."""
 import numpy as np
 import pytest

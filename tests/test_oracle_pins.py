@@ -250,7 +250,7 @@ def test_route_ties_go_to_lower_flat_index_and_classes():
 
 def test_route_per_token_topk():
     g = np.random.default_rng(9)
-    for S, K in [(4, 1), (8, 2), (16, 4)]:               # the paper's VLM grid (Appendix B.2)
+    for S, K in [(4, 1), (8, 2), (16, 4)]:               # the paper's VLM grid (Appendix C.2)
         sc = g.standard_normal((100, S)).astype(np.float32)
         rc, mask = O.route(sc, None, S, K, mode=O.MODE_PER_TOKEN)
         top = np.argsort(-sc, axis=1, kind="stable")[:, :K]
