@@ -1,17 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the sub-token-routed decode path on B200.
 
-One "step" is one pass of the whole hot path over one batch of synthetic input:
-  stc_build_page_meta -> stc_route_pack -> stc_quest_select -> stc_decode_attn
-(the write side and the read side, each once).  The metric is decode-attention
-GB/s: ALGORITHMIC bytes (what the method itself must move: keys read for the
-metadata, router scores once, kept value groups in and out, page metadata,
-selected keys, packed values, masks, offsets and page ids) divided by device
-time.  Every call is bracketed by CUDA events on the launching stream inside
-the timed region, so the line also carries per-call GB/s and the roofline
-fraction of the dominant kernel against the measured copy bandwidth.
+One "step" is one decode step over a resident compressed cache:
+  stc_quest_select -> stc_decode_attn
+(query-aware page selection, then routed attention over the selected pages), on
+synthetic inputs of the named workload; the write side (stc_build_page_meta,
+stc_route_pack) builds that cache before the timed region and is reported on its
+own (`per_call`, `full_pass`).  The metric is decode-attention GB/s: ALGORITHMIC
+bytes of the step (page metadata scanned, selected keys, packed value groups,
+masks, offsets, page ids, queries and outputs) divided by device time (CUDA
+events around K graph replays with rotating query sets).  Every call is also
+timed on its own, and `roofline` holds the dominant kernel of the step against
+the measured copy bandwidth.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4]
   python bench.py --impl reference ...       # the CPU checker, timed as it stands
 """
 from __future__ import annotations
@@ -37,7 +39,7 @@ from paper_2604_21335_b200 import workload as W  # noqa: E402
 METRIC = "decode_attention_GBps"
 UNIT = "GB/s"
 SM_SCALE = 1.0 / math.sqrt(128.0)
-FALLBACK_HBM_GBS = 6650.0        # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+FALLBACK_HBM_GBS = 6650.0        # used only when MEASURED_PEAKS.json is absent
 NOMINAL_HBM_GBS = 8000.0
 
 
@@ -125,46 +127,53 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------- CPU checker
-def oracle_step(w: W.Workload, d_cpu: dict, problems: list, q_index: int = 0) -> dict:
-    """One pass of the CPU checker over the listed (batch, kv head) problems.
-    Returns wall seconds and the same algorithmic byte count as the GPU arm."""
-    import numpy as np
-    import oracle as O
-    gq = w.gq
-    bs = sorted({b for b, _ in problems})
-    work = []
-    for b in bs:                           # slice the sample out before the clock starts
-        hs = [h for bb, h in problems if bb == b]
-        work.append(dict(
-            k=np.ascontiguousarray(d_cpu["k"][b:b + 1, hs]), v=np.ascontiguousarray(d_cpu["v"][b:b + 1, hs]),
-            sc=np.ascontiguousarray(d_cpu["scores"][b:b + 1, hs]),
-            q=np.ascontiguousarray(np.concatenate(
-                [d_cpu["q"][q_index, b:b + 1, h * gq:(h + 1) * gq] for h in hs], axis=1)),
-            cls=None if d_cpu["tok_class"] is None else d_cpu["tok_class"][b:b + 1],
-            sl=d_cpu["seq_len"][b:b + 1]))
-    t0 = time.perf_counter()
-    # one batch element at a time, so the batched drivers (OpenMP over problems) are used
-    for x in work:
-        kmin, kmax = O.page_meta_batch(x["k"], x["sl"])
-        r = O.route_pack_batch(x["v"], x["sc"], x["cls"], w.n_groups, w.k_nominal, w.t_cache * w.n_groups,
-                               x["sl"])
+class OracleSample:
+    """The CPU checker on a sample of (batch, kv head) problems, laid out as a batch of
+    one-KV-head sequences.  prepare() runs its write side once (untimed: it is not part of a decode
+    step); read_step() is one decode step (page selection + routed attention) and is what is timed."""
+
+    def __init__(self, w: W.Workload, d_cpu: dict, n_problems: int):
+        import numpy as np
+        import oracle as O
+        self.O, self.np = O, np
+        self.w = W.problem_view(w, list(range(n_problems)))      # batch = sample size, one KV head each
+        self.full = w
+        self.k, self.v = O.bf16_bits(d_cpu["k"]), O.bf16_bits(d_cpu["v"])
+        self.q = O.bf16_bits(d_cpu["q"])                           # [NQ, n, Gq, 128]
+        self.scores = d_cpu["scores"].numpy()
+        self.cls = None if d_cpu["tok_class"] is None else d_cpu["tok_class"].numpy()
+        self.seq_len = d_cpu["seq_len"].numpy()
+        self.state = None
+
+    def prepare(self):
+        O, w = self.O, self.full
+        kmin, kmax = O.page_meta_batch(self.k, self.seq_len)
+        r = O.route_pack_batch(self.v, self.scores, self.cls, w.n_groups, w.k_nominal,
+                               w.t_cache * w.n_groups, self.seq_len)
+        self.state = dict(kmin=kmin, kmax=kmax, **r)
+
+    def read_step(self, qi: int):
+        O, w, st = self.O, self.full, self.state
+        t0 = time.perf_counter()
         if w.token_budget is None:
             ids = n = None
         else:
-            ids, n = O.select_batch(x["q"], kmin, kmax, w.token_budget, w.t_cache, x["sl"])
-        O.attend_batch(x["q"], x["k"], w.n_groups, r["mask"], ids, n, SM_SCALE, packed=r["packed"],
-                       offs=r["offs"], seq_len=x["sl"])
-    dt = time.perf_counter() - t0
-    return dict(seconds=dt)
+            ids, n = O.select_batch(self.q[qi], st["kmin"], st["kmax"], w.token_budget, w.t_cache, self.seq_len)
+        out, lse = O.attend_batch(self.q[qi], self.k, w.n_groups, st["mask"], ids, n, SM_SCALE,
+                                  packed=st["packed"], offs=st["offs"], seq_len=self.seq_len)
+        return time.perf_counter() - t0, out, ids, n
+
+    def near_ties(self, qi: int, rel: float = 1e-6) -> int:
+        """Pages whose fp64 bound lies within rel*max(1,|U_k|) of the k-th largest, summed over the sample."""
+        w, st = self.full, self.state
+        if w.token_budget is None:
+            return 0
+        return int(self.O.near_ties_batch(self.q[qi], st["kmin"], st["kmax"], w.token_budget, w.t_cache,
+                                          self.seq_len, rel).sum())
 
 
-def cpu_inputs(w: W.Workload, d: dict) -> dict:
-    import oracle as O
-    out = dict(k=O.bf16_bits(d["k"].cpu()), v=O.bf16_bits(d["v"].cpu()), q=O.bf16_bits(d["q"].cpu()),
-               scores=d["scores"].cpu().numpy(),
-               tok_class=None if d["tok_class"] is None else d["tok_class"].cpu().numpy(),
-               seq_len=d["seq_len"].cpu().numpy())
-    return out
+def sample_bytes(w: W.Workload, n_problems: int, ab_read: int) -> float:
+    return ab_read * n_problems / w.n_problems
 
 
 # ------------------------------------------------------------------------ GPU arm
@@ -189,6 +198,41 @@ def sample_problems(w: W.Workload, n: int):
     return [allp[int(i * stride)] for i in range(n)]
 
 
+def workload_string(w: W.Workload) -> str:
+    return (f"{w.name}: B{w.batch} Hq{w.n_q_heads} Hkv{w.n_kv_heads} T{w.t_cache} S{w.n_groups} "
+            f"keep{w.k_nominal} budget{w.token_budget}, one decode step per step "
+            "(stc_quest_select + stc_decode_attn over the resident compressed cache)")
+
+
+L2_BYTES = 126 << 20
+NQ = 8                                                      # rotating query sets
+
+
+def read_bytes_estimate(w: W.Workload) -> int:
+    """Shape-only estimate of a decode step's algorithmic bytes (sizes the number of cache copies)."""
+    sel = w.n_pages if w.token_budget is None else min(w.n_pages, w.token_budget // 16)
+    per = sel * 16 * (256 + w.k_nominal * w.group_dim * 2 + 2)
+    if w.token_budget is not None:
+        per += w.n_pages * 512
+    return per * w.n_problems
+
+
+class Copy:
+    """One resident cache (inputs, compressed store, write-side workspaces)."""
+
+    def __init__(self, P, Bd, w, dev, seed):
+        self.w = W.shrink(w, seed=seed)
+        self.d = W.make_inputs(self.w, dev, n_queries=NQ)
+        B, Hkv, Hq, T, S = w.batch, w.n_kv_heads, w.n_q_heads, w.t_cache, w.n_groups
+        self.shape = P.Shape(B, Hq, Hkv, S, T, self.d["seq_len"])
+        self.cap = (T - w.n_text) * w.k_nominal + w.n_text * S
+        self.cache = P.Cache.allocate(self.shape, self.d["k"], self.cap)
+        self.total = torch.zeros(B, Hkv, dtype=torch.int64, device=dev)
+        self.status = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
+        self.ws_r = Bd.new_workspace(self.shape, Bd.OP_ROUTE_PACK, device=dev)
+        self.qs = [self.d["q"][i].contiguous() for i in range(NQ)]
+
+
 def run_gpu(args, r: D.Rank):
     import paper_2604_21335_b200 as P
     from paper_2604_21335_b200 import binding as Bd
@@ -196,81 +240,89 @@ def run_gpu(args, r: D.Rank):
     torch.cuda.set_device(dev)
     P.load_library()                       # fails loudly if the CUDA library is missing
     w = select_workload(args)
-    w = W.shrink(w, seed=w.seed + 7919 * r.rank)          # each rank owns its own batch (weak scaling)
-    NQ = 8
-    d = W.make_inputs(w, dev, n_queries=NQ)
     B, Hkv, Hq, T, S = w.batch, w.n_kv_heads, w.n_q_heads, w.t_cache, w.n_groups
-    shape = P.Shape(B, Hq, Hkv, S, T, d["seq_len"])
-    n_full_tokens = w.n_text
-    cap = (T - n_full_tokens) * w.k_nominal + n_full_tokens * S
-    cache = P.Cache.allocate(shape, d["k"], cap)
-    total = torch.zeros(B, Hkv, dtype=torch.int64, device=dev)
-    status = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
-    out = torch.zeros(B, Hq, 128, dtype=torch.float32, device=dev)
+    # Decode steps whose working set fits L2 would be served from L2 by the second step: such
+    # workloads rotate independent cache copies (one per query set) so that consecutive steps
+    # touch different lines; larger ones use one cache and rotate the queries only.
+    n_copies = 1 if read_bytes_estimate(w) >= 2 * L2_BYTES else NQ
+    copies = [Copy(P, Bd, w, dev, w.seed + 7919 * r.rank + 104729 * c) for c in range(n_copies)]
+    shape = copies[0].shape
     if w.token_budget is None:
-        page_ids = n_pages = None
         max_pages = shape.n_pages
+        ids = npg = [None] * NQ
     else:
         max_pages = max(1, min(shape.n_pages, w.token_budget // 16))
-        page_ids = torch.zeros(B, Hkv, max_pages, dtype=torch.int32, device=dev)
-        n_pages = torch.zeros(B, Hkv, dtype=torch.int32, device=dev)
-    ws_r = Bd.new_workspace(shape, Bd.OP_ROUTE_PACK, device=dev)
+        ids = [torch.zeros(B, Hkv, max_pages, dtype=torch.int32, device=dev) for _ in range(NQ)]
+        npg = [torch.zeros(B, Hkv, dtype=torch.int32, device=dev) for _ in range(NQ)]
+    out = torch.zeros(B, Hq, 128, dtype=torch.float32, device=dev)
     ws_s = Bd.new_workspace(shape, Bd.OP_QUEST_SELECT, device=dev)
     ws_a = Bd.new_workspace(shape, Bd.OP_DECODE_ATTN, max_pages, device=dev)
-    qs = [d["q"][i].contiguous() for i in range(NQ)]
     names = ["page_meta", "route_mask", "pack_values", "quest_select", "decode_attn"]
-    launches_per_step = 1 + 2 + (1 if page_ids is not None else 0) + 1   # route_pack = select kernel + compact kernel
-
-    # The key side (page metadata, page selection) and the value side (routing, packing) of a
-    # pass touch disjoint data, so they run on two streams and join before the attention call;
-    # --serial puts all five calls on one stream.
     side = None if args.serial else torch.cuda.Stream(device=dev)
 
-    def value_side():
-        P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)     # stc_route_pack, first half
-        P.pack_values(shape, d["v"], cache, total, status, ws_r)                       # ... second half
+    def copy_of(j):
+        return copies[j % n_copies]
 
-    def step(i):
-        q = qs[i % NQ]
+    def value_side(c):
+        P.route_mask(c.shape, c.d["scores"], c.d["tok_class"], w.k_nominal, c.cache, c.ws_r)
+        P.pack_values(c.shape, c.d["v"], c.cache, c.total, c.status, c.ws_r)
+
+    def write_side(j):
+        # the key side (page metadata) and the value side (routing, packing) touch disjoint data:
+        # two streams, joined at the end; --serial keeps one stream
+        c = copy_of(j)
         main = torch.cuda.current_stream()
         if side is not None:
             side.wait_stream(main)
             with torch.cuda.stream(side):
-                value_side()
-        P.build_page_meta(shape, cache)
+                value_side(c)
+        P.build_page_meta(c.shape, c.cache)
         if side is None:
-            value_side()
-        if page_ids is not None:
-            P.quest_select(shape, cache, q, w.token_budget, page_ids, n_pages, ws_s)
-        if side is not None:
+            value_side(c)
+        else:
             main.wait_stream(side)
-        P.decode_attn(shape, cache, q, page_ids, n_pages, SM_SCALE, out, ws_a)
 
+    def read_step(j):
+        c = copy_of(j)
+        if ids[j] is not None:
+            P.quest_select(c.shape, c.cache, c.qs[j], w.token_budget, ids[j], npg[j], ws_s)
+        P.decode_attn(c.shape, c.cache, c.qs[j], ids[j], npg[j], SM_SCALE, out, ws_a)
+
+    # ---- build the resident caches (the write side; also its warm-up), then warm the read side --
     W_ = max(args.warmup, 3)
-    for i in range(W_):
-        step(i)
+    for c in range(n_copies):
+        write_side(c)
+    for i in range(max(W_, NQ)):
+        read_step(i % NQ)
     torch.cuda.synchronize()
-    assert int(status.abs().sum()) == 0, "device status reported an error"
+    for c in copies:
+        assert int(c.status.abs().sum()) == 0, "device status reported an error"
     assert int(ws_a[:4].view(torch.int32)[0]) == 0, "stc_decode_attn device status"
 
-    # algorithmic bytes from what the step actually kept / selected
-    seq = d["seq_len"].cpu().tolist()
-    cnt = torch.zeros_like(cache.v_mask, dtype=torch.int32)
-    for j in range(S):
-        cnt += (cache.v_mask.int() >> j) & 1
-    if page_ids is not None:
-        tok_idx = (page_ids.long()[..., None] * 16 + torch.arange(16, device=dev)).flatten(2)
-        valid = tok_idx < d["seq_len"].long()[:, None, None]
-        sel_groups = int((torch.gather(cnt, 2, tok_idx.clamp(max=T - 1)) * valid).sum())
-        sel_tokens, sel_pages = int(valid.sum()), int(n_pages.sum())
-    else:
-        sel_groups, sel_tokens = int(cnt.sum()), int(sum(seq)) * Hkv
-        sel_pages = int(sum((n + 15) // 16 for n in seq)) * Hkv
-    del cnt
-    n_routed = (int(sum(seq)) - n_full_tokens * B) * Hkv
-    ab = algorithmic_bytes(w, seq, n_routed, n_full_tokens * B * Hkv, int(total.sum()), sel_pages,
-                           sel_tokens, sel_groups)
-    step_bytes = sum(ab.values())
+    # ---- algorithmic bytes from what the steps actually kept / selected (mean over the query sets)
+    seq = copies[0].d["seq_len"].cpu().tolist()
+    n_routed = (int(sum(seq)) - w.n_text * B) * Hkv
+    abs_ = []
+    for j in range(NQ):
+        c = copy_of(j)
+        cnt = torch.zeros_like(c.cache.v_mask, dtype=torch.int32)
+        for g_ in range(S):
+            cnt += (c.cache.v_mask.int() >> g_) & 1
+        if ids[j] is not None:
+            tok_idx = (ids[j].long()[..., None] * 16 + torch.arange(16, device=dev)).flatten(2)
+            valid = tok_idx < c.d["seq_len"].long()[:, None, None]
+            sel_groups = int((torch.gather(cnt, 2, tok_idx.clamp(max=T - 1)) * valid).sum())
+            sel_tokens, sel_pages = int(valid.sum()), int(npg[j].sum())
+        else:
+            sel_groups, sel_tokens = int(cnt.sum()), int(sum(seq)) * Hkv
+            sel_pages = int(sum((n + 15) // 16 for n in seq)) * Hkv
+        del cnt
+        abs_.append((algorithmic_bytes(w, seq, n_routed, w.n_text * B * Hkv, int(c.total.sum()), sel_pages,
+                                       sel_tokens, sel_groups), sel_tokens))
+    ab = {n: sum(a[n] for a, _ in abs_) // NQ for n in names}
+    sel_tokens = sum(t for _, t in abs_) // NQ
+    read_bytes = ab["quest_select"] + ab["decode_attn"]
+    pass_bytes = sum(ab.values())
 
     # ---- one CUDA graph per query set: a step is one graph launch, so the timed region holds
     #      device work only (a Python-driven launch sequence is CPU-bound on the small workloads)
@@ -282,18 +334,18 @@ def run_gpu(args, r: D.Rank):
 
     launch_mode = "cuda_graph"
     try:
-        step_graphs = [capture(lambda j=j: step(j)) for j in range(NQ)]
+        step_graphs = [capture(lambda j=j: read_step(j)) for j in range(NQ)]
         run_step = lambda i: step_graphs[i % NQ].replay()
     except Exception as e:                                   # noqa: BLE001
         if r.is_main:
             print(f"# graph capture unavailable ({type(e).__name__}: {e}); timing eager launches", file=sys.stderr)
         launch_mode = "eager"
-        run_step = step
-    for i in range(W_):
+        run_step = lambda i: read_step(i % NQ)
+    for i in range(max(W_, NQ)):
         run_step(i)
     torch.cuda.synchronize()
 
-    # ---- timed region: exactly K steps -----------------------------------------------------------
+    # ---- timed region: exactly K decode steps ----------------------------------------------------
     K = args.steps
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(dev.index or 0)
@@ -309,68 +361,129 @@ def run_gpu(args, r: D.Rank):
     D.barrier(r)
     total_ms = D.max_over_ranks(r, ev0.elapsed_time(ev1))
     ms_per_step = total_ms / K
-    value = step_bytes * r.world / (ms_per_step * 1e-3) / 1e9
+    value = read_bytes * r.world / (ms_per_step * 1e-3) / 1e9
 
-    # ---- each call on its own: NQ back-to-back launches (rotating queries) per graph replay -------
-    def call_fn(c, j):
-        q = qs[j]
-        if c == 0:
-            P.build_page_meta(shape, cache)
-        elif c == 1:
-            P.route_mask(shape, d["scores"], d["tok_class"], w.k_nominal, cache, ws_r)
-        elif c == 2:
-            P.pack_values(shape, d["v"], cache, total, status, ws_r)
-        elif c == 3:
-            if page_ids is not None:
-                P.quest_select(shape, cache, q, w.token_budget, page_ids, n_pages, ws_s)
-        else:
-            P.decode_attn(shape, cache, q, page_ids, n_pages, SM_SCALE, out, ws_a)
-
-    per_call_ms = []
-    for c in range(5):
-        if c == 3 and page_ids is None:
-            per_call_ms.append(0.0)
-            continue
-        body = lambda c=c: [call_fn(c, j) for j in range(NQ)]
-        if launch_mode == "cuda_graph":
-            g = capture(body)
-            run = g.replay
-        else:
-            run = body
+    def timed(run, reps):
         run()
         torch.cuda.synchronize()
-        reps = max(2, min(50, int(20.0 / max(ms_per_step * NQ, 1e-3))))
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(reps):
             run()
         e1.record()
         torch.cuda.synchronize()
-        per_call_ms.append(e0.elapsed_time(e1) / (reps * NQ))
-    if page_ids is not None:                                  # the last select ran with query NQ-1: redo the step's
-        step(0)
+        return e0.elapsed_time(e1) / reps
+
+    def graphed(body):
+        if launch_mode == "cuda_graph":
+            return capture(body).replay
+        return body
+
+    # ---- each call on its own: NQ back-to-back launches per graph replay, query set j on its own
+    #      cache copy and (decode_attn) with the page list that query selected ------------------------
+    def call_fn(cidx, j):
+        c = copy_of(j)
+        if cidx == 0:
+            P.build_page_meta(c.shape, c.cache)
+        elif cidx == 1:
+            P.route_mask(c.shape, c.d["scores"], c.d["tok_class"], w.k_nominal, c.cache, c.ws_r)
+        elif cidx == 2:
+            P.pack_values(c.shape, c.d["v"], c.cache, c.total, c.status, c.ws_r)
+        elif cidx == 3:
+            P.quest_select(c.shape, c.cache, c.qs[j], w.token_budget, ids[j], npg[j], ws_s)
+        else:
+            P.decode_attn(c.shape, c.cache, c.qs[j], ids[j], npg[j], SM_SCALE, out, ws_a)
+
+    budget_ms = 400.0                                        # device time spent on each extra measurement
+    per_call_ms = []
+    for cidx in range(5):
+        if cidx == 3 and ids[0] is None:
+            per_call_ms.append(0.0)
+            continue
+        run = graphed(lambda cidx=cidx: [call_fn(cidx, j) for j in range(NQ)])
+        est = ms_per_step * NQ * (8.0 if cidx < 3 else 1.0)
+        per_call_ms.append(timed(run, max(2, min(50, int(budget_ms / max(est, 1e-3))))) / NQ)
+
+    # ---- the whole pass (write side + decode step), as an extra figure ---------------------------
+    run = graphed(lambda: [(write_side(j), read_step(j)) for j in range(NQ)])
+    pass_ms = timed(run, max(1, min(20, int(budget_ms / max(sum(per_call_ms) * NQ, 1e-3))))) / NQ
+    torch.cuda.synchronize()
+    for c in copies:
+        assert int(c.status.abs().sum()) == 0
+
+    # ---- the CPU checker on a sample of problems: timed baseline, parity check, near-tie count ----
+    probs = sample_problems(w, args.cpu_problems)
+    cpu_baseline = checked = None
+    oracle_out = None
+    if r.world == 1 and not args.no_cpu:
+        import numpy as np
+        import oracle as O
+        c0 = copies[0]
+        d_cpu = dict(k=torch.stack([c0.d["k"][b, h:h + 1] for b, h in probs]).cpu(),
+                     v=torch.stack([c0.d["v"][b, h:h + 1] for b, h in probs]).cpu(),
+                     scores=torch.stack([c0.d["scores"][b, h:h + 1] for b, h in probs]).cpu(),
+                     q=torch.stack([c0.d["q"][:, b, h * w.gq:(h + 1) * w.gq] for b, h in probs], dim=1).cpu(),
+                     tok_class=None if c0.d["tok_class"] is None else
+                     torch.stack([c0.d["tok_class"][b] for b, _ in probs]).cpu(),
+                     seq_len=torch.stack([c0.d["seq_len"][b] for b, _ in probs]).cpu())
+        smp = OracleSample(c0.w, d_cpu, len(probs))
+        smp.prepare()
+        smp.read_step(0)                                       # page in the library
+        secs, oracle_out = 0.0, None
+        for qi in range(NQ):
+            if n_copies > 1 and qi > 0:
+                break                                          # other query sets belong to other cache copies
+            dt, o_out, o_ids, o_n = smp.read_step(qi)
+            secs += dt
+            if qi == 0:
+                oracle_out, oracle_ids, oracle_n = o_out, o_ids, o_n
+        n_steps_cpu = 1 if n_copies > 1 else NQ
+        cpu_baseline = {"value": round(sample_bytes(w, len(probs), read_bytes) * n_steps_cpu / secs / 1e9, 4),
+                        "unit": UNIT, "cores": O.n_threads(), "kind": "oracle",
+                        "sample": f"{n_steps_cpu} decode step(s) over {len(probs)} of {w.n_problems} "
+                                  f"(batch, kv head) problems, {secs:.2f} s (its write side, untimed, ran once)",
+                        "tokens_heads_per_s_context": round(len(probs) * w.gq * T * n_steps_cpu / secs)}
+
+        def sample_err(o_t):                                    # [B,Hq,128] tensor vs the checker's sample
+            got = torch.stack([o_t[b, h * w.gq:(h + 1) * w.gq] for b, h in probs]).double().cpu().numpy()
+            diff = np.abs(got - oracle_out)
+            return float(diff.max()), float(diff.mean() / max(np.abs(oracle_out).mean(), 1e-30))
+
+        read_step(0)
         torch.cuda.synchronize()
+        ma, mr = sample_err(out)
+        assert ma <= 1e-2 and mr <= 2e-3, ("device-resident decode step vs CPU checker", ma, mr)
+        if ids[0] is not None:
+            for i, (b, h) in enumerate(probs):
+                assert int(npg[0][b, h]) == int(oracle_n[i, 0])
+                assert np.array_equal(ids[0][b, h, :int(oracle_n[i, 0])].cpu().numpy(),
+                                      oracle_ids[i, 0, :int(oracle_n[i, 0])]), "page ids differ from the CPU checker"
+        checked = {"problems": len(probs), "page_ids": "bit-exact" if ids[0] is not None else "selection off",
+                   "decode_step": {"max_abs": ma, "mean_rel": mr},
+                   "near_tie_pages_1e-6": smp.near_ties(0)}
 
     # ---- end to end through the C-ABI with host buffers ----------------------------
-    e2e = None
+    e2e = e2e_pass = None
     if not args.no_e2e:
-        hk = d["k"].cpu().pin_memory(); hv = d["v"].cpu().pin_memory()
-        hs = d["scores"].cpu().pin_memory()
-        hc = None if d["tok_class"] is None else d["tok_class"].cpu().pin_memory()
-        hq = [q.cpu().pin_memory() for q in qs]
+        c0 = copies[0]
+        hq = [q.cpu().pin_memory() for q in c0.qs]
         h_out = torch.zeros(B, Hq, 128, dtype=torch.float32).pin_memory()
-        h_tot = torch.zeros(B, Hkv, dtype=torch.int64).pin_memory()
-        h_st = torch.zeros(B, Hkv, dtype=torch.int32).pin_memory()
-        arena = torch.empty(Bd.pass_host_arena_bytes(shape, cap, w.token_budget), dtype=torch.uint8, device=dev)
+        h_st = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+        arena = torch.empty(Bd.decode_step_host_arena_bytes(shape, w.token_budget), dtype=torch.uint8, device=dev)
         Ke = max(1, min(K, args.e2e_steps))
 
-        def e2e_step(i):
-            Bd.pass_host(shape, hk, hv, hs, hc, hq[i % NQ], w.token_budget, w.k_nominal, SM_SCALE, cap,
-                         arena, h_out, h_tot, h_st)
+        def e2e_step(i):                                    # the cache stays resident; the query comes from the host
+            Bd.decode_step_host(shape, c0.cache, hq[i % NQ], w.token_budget, SM_SCALE, arena, h_out, h_st)
             torch.cuda.current_stream().synchronize()      # the step's result is read on the host
             return float(h_out[0, 0, 0])
 
-        for i in range(2):
+        e2e_step(0)
+        assert int(h_st[0]) == 0
+        if oracle_out is not None:                          # same result as the checker before anything is timed
+            ma, mr = sample_err(h_out)
+            assert ma <= 1e-2 and mr <= 2e-3, ("stc_decode_step_host vs CPU checker", ma, mr)
+            checked["decode_step_host"] = {"max_abs": ma, "mean_rel": mr}
+        for i in range(3):
             e2e_step(i)
         D.barrier(r)
         torch.cuda.synchronize()
@@ -378,69 +491,94 @@ def run_gpu(args, r: D.Rank):
         for i in range(Ke):
             e2e_step(i)
         torch.cuda.synchronize()
-        e2e_ms = (time.perf_counter() - t0) * 1e3 / Ke
-        e2e_ms = D.max_over_ranks(r, e2e_ms)
-        assert int(h_st.abs().sum()) == 0
-        # same result as the device-resident path (same query as the last timed step there)
-        h2d = hk.numel() * 2 + hv.numel() * 2 + hs.numel() * 4 + (0 if hc is None else hc.numel()) + hq[0].numel() * 2
-        d2h = h_out.numel() * 4 + h_tot.numel() * 8 + h_st.numel() * 4
-        e2e = {"value": step_bytes * r.world / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
-               "steps": Ke, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-        del hk, hv, hs, arena
+        e2e_ms = D.max_over_ranks(r, (time.perf_counter() - t0) * 1e3 / Ke)
+        e2e = {"value": read_bytes * r.world / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+               "steps": Ke, "h2d_bytes_per_step": hq[0].numel() * 2, "d2h_bytes_per_step": h_out.numel() * 4 + 4,
+               "call": "stc_decode_step_host (query from pinned host memory, selection + attention on the "
+                       "resident cache, result back to the host)"}
+        del arena
+
+        if not args.no_e2e_pass:
+            # the whole pass from host buffers (keys, values and scores cross PCIe every step)
+            hk = c0.d["k"].cpu().pin_memory(); hv = c0.d["v"].cpu().pin_memory()
+            hs = c0.d["scores"].cpu().pin_memory()
+            hc = None if c0.d["tok_class"] is None else c0.d["tok_class"].cpu().pin_memory()
+            h_tot = torch.zeros(B, Hkv, dtype=torch.int64).pin_memory()
+            h_stp = torch.zeros(B, Hkv, dtype=torch.int32).pin_memory()
+            arena = torch.empty(Bd.pass_host_arena_bytes(shape, c0.cap, w.token_budget), dtype=torch.uint8, device=dev)
+            h2d = hk.numel() * 2 + hv.numel() * 2 + hs.numel() * 4 + (0 if hc is None else hc.numel()) + hq[0].numel() * 2
+            Kp = max(1, min(Ke, int(2e10 // h2d) or 1, 20))
+
+            def pass_step(i):
+                Bd.pass_host(shape, hk, hv, hs, hc, hq[i % NQ], w.token_budget, w.k_nominal, SM_SCALE, c0.cap,
+                             arena, h_out, h_tot, h_stp)
+                torch.cuda.current_stream().synchronize()
+
+            pass_step(0)
+            assert int(h_stp.abs().sum()) == 0
+            if oracle_out is not None:
+                ma, mr = sample_err(h_out)
+                assert ma <= 1e-2 and mr <= 2e-3, ("stc_pass_host vs CPU checker", ma, mr)
+                checked["pass_host"] = {"max_abs": ma, "mean_rel": mr}
+            t0 = time.perf_counter()
+            for i in range(Kp):
+                pass_step(i)
+            torch.cuda.synchronize()
+            p_ms = D.max_over_ranks(r, (time.perf_counter() - t0) * 1e3 / Kp)
+            e2e_pass = {"value": pass_bytes * r.world / (p_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": p_ms,
+                        "steps": Kp, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": h_out.numel() * 4 + h_tot.numel() * 8 + h_stp.numel() * 4,
+                        "call": "stc_pass_host (whole pass from pinned host buffers)"}
+            del hk, hv, hs, arena
 
     if not r.is_main:
         return
     peak, peak_src = peaks()
     per_kernel = {}
-    for c, n in enumerate(names):
-        ms = per_call_ms[c]
+    for cidx, n in enumerate(names):
+        ms = per_call_ms[cidx]
         gbs = ab[n] / (ms * 1e-3) / 1e9 if ms > 0 and ab[n] else 0.0
         per_kernel[n] = {"us": round(ms * 1e3, 2), "alg_bytes": ab[n], "GBps": round(gbs, 1),
                          "frac_of_" + peak_src: round(gbs / peak, 4), "frac_of_8TBps": round(gbs / NOMINAL_HBM_GBS, 4)}
-    read_ms = per_call_ms[3] + per_call_ms[4]
-    read_bytes = ab["quest_select"] + ab["decode_attn"]
-    read_gbs = read_bytes / (read_ms * 1e-3) / 1e9
-    # dominant call of the step (every call is one kernel)
-    single = {n: per_call_ms[c] for c, n in enumerate(names) if ab[n]}
-    dom = max(single, key=single.get)
-    kernel_of = dict(KERNEL_OF)
-    if (T + 255) // 256 <= 32 // S:                      # problems that fit one CTA take the small selection kernel
-        kernel_of["route_mask"] = "route_select_small_kernel"
-    roof = {"bound": "hbm", "kernel": kernel_of[dom], "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
+    # dominant kernel of the timed step (each call of the step is one kernel)
+    step_calls = {n: per_call_ms[names.index(n)] for n in ("quest_select", "decode_attn") if ab[n]}
+    dom = max(step_calls, key=step_calls.get)
+    traffic = TRAFFIC_NOTE.get((w.name, w.batch, w.token_budget, w.k_nominal, dom))
+    roof = {"bound": "hbm", "kernel": KERNEL_OF[dom] + (f"<{w.gq}>" if dom == "quest_select" else ""),
+            "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
             "frac": round(per_kernel[dom]["GBps"] / peak, 4), "peak_source": peak_src + " copy bandwidth",
-            "traffic": TRAFFIC_NOTE.get((args.workload, dom))}
+            "traffic": traffic}
+    ws_mib = read_bytes / 2 ** 20
+    if n_copies == 1:
+        l2 = ("a decode step moves %.0f MiB (larger than L2, page metadata re-read every step); %d rotating query "
+              "sets, each with its own page list" % (ws_mib, NQ))
+    else:
+        l2 = ("a decode step moves %.0f MiB (fits L2): %d independent cache copies rotate with the query sets, so "
+              "consecutive steps touch different lines (%.0f MiB per rotation)" % (ws_mib, n_copies, ws_mib * n_copies))
+    if ws_mib * n_copies < 2 * L2_BYTES / 2 ** 20:
+        l2 += "; L2-assisted: the rotation is smaller than twice L2"
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": r.world, "steps": K,
-        "warmup": W_, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "warmup": max(W_, NQ), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{w.name}: B{B} Hq{Hq} Hkv{Hkv} T{T} S{S} keep{w.k_nominal} "
-                               f"budget{w.token_budget}, one full pass per step "
-                               "(page_meta + route_pack + quest_select + decode_attn)",
-                   "l2": "inputs larger than L2 (K+V %.0f MiB re-read every step), %d rotating query sets"
-                         % ((d["k"].numel() + d["v"].numel()) * 2 / 2 ** 20, NQ),
-                   "replicas": "one independent batch per rank, no collective",
-                   "streams": "one" if args.serial else "two (key side | value side, joined before decode_attn)"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "launch": launch_mode,
+        "config": {"workload": workload_string(w), "l2": l2,
+                   "replicas": "one independent batch per rank, no collective"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": (2 if ids[0] is not None else 1) * K, "launch": launch_mode,
         "roofline": roof,
+        "frac_of_" + peak_src: round(value / r.world / peak, 4), "frac_of_8TBps": round(value / r.world / NOMINAL_HBM_GBS, 4),
         "per_call": per_kernel,
-        "read_side": {"us": round(read_ms * 1e3, 2), "alg_bytes": read_bytes, "GBps": round(read_gbs, 1),
-                      "frac_of_" + peak_src: round(read_gbs / peak, 4),
-                      "frac_of_8TBps": round(read_gbs / NOMINAL_HBM_GBS, 4)},
+        "read_side": {"us": round(ms_per_step * 1e3, 2), "alg_bytes": read_bytes, "GBps": round(value / r.world, 1),
+                      "sum_of_calls_us": round((per_call_ms[3] + per_call_ms[4]) * 1e3, 2)},
+        "full_pass": {"us": round(pass_ms * 1e3, 2), "alg_bytes": pass_bytes,
+                      "GBps": round(pass_bytes / (pass_ms * 1e-3) / 1e9, 1),
+                      "streams": "one" if args.serial else "two (page metadata | routing + packing, joined before the decode step)"},
+        "e2e_full_pass": e2e_pass,
         "tokens_heads_per_s": {"context": round(B * Hq * T * r.world / (ms_per_step * 1e-3)),
                                "attended": round(sel_tokens * w.gq * r.world / (ms_per_step * 1e-3))},
     }
-    if r.world == 1 and not args.no_cpu:
-        dc = cpu_inputs(w, d)
-        probs = sample_problems(w, args.cpu_problems)
-        import oracle as O
-        oracle_step(w, dc, probs[:1])                          # page in the library
-        res = oracle_step(w, dc, probs)
-        frac = len(probs) / w.n_problems
-        line["cpu_baseline"] = {"value": round(step_bytes * frac / res["seconds"] / 1e9, 4), "unit": UNIT,
-                                "cores": O.n_threads(), "kind": "oracle",
-                                "sample": f"one full pass over {len(probs)} of {w.n_problems} (batch, kv head) "
-                                          f"problems, {res['seconds']:.2f} s",
-                                "tokens_heads_per_s_context": round(len(probs) * w.gq * T / res["seconds"])}
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
+        line["checked_against_cpu"] = checked
     print(json.dumps(line), flush=True)
 
 
@@ -448,12 +586,10 @@ KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kern
              "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel",
              "route_mask": "route_select_kernel"}
 
-# Per-launch DRAM traffic of the dominant kernel from the committed ncu capture
-# (profiles/), in bytes; None until a capture exists for that workload.
+# Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes) of the step's dominant
+# kernel from the committed ncu captures under profiles/, keyed by (workload, batch, budget, keep, call);
+# absent = no capture of the kernel as it stands.
 TRAFFIC_NOTE: dict = {
-    # route_compact_kernel on this very workload: dram__bytes_read 205.7 MB + dram__bytes_write 83.0 MB per launch
-    # (profiles/traffic_bench_cfg1.md; part of the packed store is still in L2 when the kernel ends)
-    ("cfg1", "pack_values"): 288.5e6,
 }
 
 
@@ -510,19 +646,20 @@ def run_router(args):
 
 # -------------------------------------------------------------------- reference arm
 def run_reference(args, r: D.Rank):
+    """The CPU checker as it stands on a sample of the same workload: its write side once
+    (untimed), then K decode steps (page selection + routed attention) with rotating queries."""
     if not r.is_main:
         return
     import oracle as O
     w = select_workload(args)
-    d = W.make_inputs(w, "cpu", n_queries=8)
-    dc = cpu_inputs(w, d)
     probs = sample_problems(w, args.cpu_problems)
-    frac = len(probs) / w.n_problems
-    seq = dc["seq_len"].tolist()
+    d = W.make_inputs(w, "cpu", n_queries=NQ, problems=probs)       # the same bits the GPU arm draws
+    smp = OracleSample(w, d, len(probs))
+    smp.prepare()
     # bytes of the sample, with the selected / kept counts the configuration implies
-    n_full = w.n_text
-    n_routed = (sum(seq) - n_full * w.batch) * w.n_kv_heads
-    total_groups = n_routed * w.k_nominal + n_full * w.batch * w.n_kv_heads * w.n_groups
+    seq = [w.t_cache] * w.batch
+    n_routed = (sum(seq) - w.n_text * w.batch) * w.n_kv_heads
+    total_groups = n_routed * w.k_nominal + w.n_text * w.batch * w.n_kv_heads * w.n_groups
     pages = sum((n + 15) // 16 for n in seq) * w.n_kv_heads
     if w.token_budget is None:
         sel_pages, sel_tokens = pages, sum(seq) * w.n_kv_heads
@@ -531,22 +668,19 @@ def run_reference(args, r: D.Rank):
         sel_tokens = sel_pages * 16
     sel_groups = int(sel_tokens * total_groups / max(1, sum(seq) * w.n_kv_heads))
     ab = algorithmic_bytes(w, seq, n_routed, 0, total_groups, sel_pages, sel_tokens, sel_groups)
-    step_bytes = sum(ab.values()) * frac
+    step_bytes = sample_bytes(w, len(probs), ab["quest_select"] + ab["decode_attn"])
     for i in range(max(args.warmup, 1)):
-        oracle_step(w, dc, probs[:max(1, len(probs) // 4)], i % 8)
+        smp.read_step(i % NQ)
     K = args.steps
-    t0 = time.perf_counter()
-    for i in range(K):
-        oracle_step(w, dc, probs, i % 8)
-    sec = (time.perf_counter() - t0) / K
+    sec = sum(smp.read_step(i % NQ)[0] for i in range(K)) / K
     value = step_bytes / sec / 1e9
-    sample = f"one full pass over {len(probs)} of {w.n_problems} (batch, kv head) problems per step"
+    sample = (f"one decode step over {len(probs)} of {w.n_problems} (batch, kv head) problems per step "
+              "(its write side, untimed, ran once)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
         "steps": K, "warmup": max(args.warmup, 1), "ms_per_step": round(sec * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{w.name}: B{w.batch} Hq{w.n_q_heads} Hkv{w.n_kv_heads} T{w.t_cache} "
-                               f"S{w.n_groups} keep{w.k_nominal} budget{w.token_budget}, CPU checker"},
+        "config": {"workload": workload_string(w)},
         "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": O.n_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -560,23 +694,24 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1", choices=sorted(W.CONFIGS))
+    ap.add_argument("--workload", default="cfg4", choices=sorted(W.CONFIGS))
     ap.add_argument("--budget", type=int, default=None, help="override the Quest token budget")
     ap.add_argument("--keep", type=int, default=None, help="override the average groups kept")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--context", type=int, default=None)
     ap.add_argument("--cpu-problems", type=int, default=None, help="problems in the CPU-checker sample")
-    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--e2e-steps", type=int, default=100)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-e2e-pass", action="store_true", help="skip the whole pass from host buffers")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--serial", action="store_true", help="all calls of a step on one stream")
+    ap.add_argument("--serial", action="store_true", help="the write side of the full pass on one stream")
     ap.add_argument("--only", default=None, choices=["router"], help="time one extra kernel instead of the step")
     args = ap.parse_args()
     if args.impl == "reference":
-        args.steps = 3 if args.steps is None else args.steps
+        args.steps = 16 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         if args.cpu_problems is None:
-            args.cpu_problems = 32
+            args.cpu_problems = 8
         world = int(os.environ.get("WORLD_SIZE", "1"))
         rank = int(os.environ.get("RANK", "0"))
         if world > 1 and rank != 0:
@@ -588,10 +723,10 @@ def main():
         args.warmup = 3 if args.warmup is None else args.warmup
         run_router(args)
         return
-    args.steps = 300 if args.steps is None else args.steps
-    args.warmup = 5 if args.warmup is None else args.warmup
+    args.steps = 2000 if args.steps is None else args.steps
+    args.warmup = 8 if args.warmup is None else args.warmup
     if args.cpu_problems is None:
-        args.cpu_problems = 32
+        args.cpu_problems = 16
     r = D.init_from_env()
     try:
         run_gpu(args, r)

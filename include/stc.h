@@ -122,7 +122,16 @@ int32_t stc_build_page_meta(const stc_shape* shape, const stc_cache* cache,
  * min(ceil(t_cap/16), token_budget/16).
  * scores_opt (may be NULL): f32 [B][Hkv][P], receives U for the valid pages.
  * Non-finite scores are not supported (selection then is unspecified, still
- * in bounds).  ws: STC_OP_QUEST_SELECT. */
+ * in bounds).  ws: STC_OP_QUEST_SELECT.  The first int32 of ws is a device
+ * status word the call writes: STC_OK, or STC_ERR_TIMEOUT if a bounded wait for
+ * an asynchronous copy expired on the device (it never should; the page lists
+ * then hold valid but unspecified ids).  It can be read after the stream has
+ * been synchronised.
+ * With several query heads per KV head and scores_opt == NULL the pages are
+ * first scored on the tensor cores (same products, another summation order) and
+ * only the pages whose approximate score lies within a rigorous error margin of
+ * the k_pg-th score are re-scored in the fixed order above; the ids written are
+ * the same either way. */
 int32_t stc_quest_select(const stc_shape* shape, const stc_cache* cache, const void* q,
                          int32_t token_budget, int32_t max_pages, int32_t* page_ids,
                          int32_t* n_pages, float* scores_opt, void* ws, size_t ws_bytes,
@@ -170,6 +179,19 @@ int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, 
 int32_t stc_quest_select_static(const stc_shape* shape, const stc_cache* cache, const void* q,
                                 int32_t token_budget, int32_t max_pages, int32_t* page_ids,
                                 int32_t* n_pages, float* scores_opt, void* stream);
+
+/* Token classes from a page selection, for running the two stages in the
+ * paper's own order (Section 3.4 / Appendix B.1: the value-group router acts on
+ * the tokens Stage I retained, with M = N*K over those N tokens):
+ *     tok_class[b][hk][t] = STC_CLS_ROUTED if a listed page of problem (b, hk)
+ *                           holds the valid token t, STC_CLS_DROP otherwise.
+ * Feeding the result to stc_route_pack (class_head_stride = t_cap) routes and
+ * packs only the selected tokens; stc_decode_attn with the same page list then
+ * attends them.  page_ids / n_pages / max_pages as written by stc_quest_select
+ * (ids outside the sequence are ignored).  tok_class: u8 [B][Hkv][t_cap], every
+ * byte is written.  Needs no workspace. */
+int32_t stc_pages_to_class(const stc_shape* shape, const int32_t* page_ids, const int32_t* n_pages,
+                           int32_t max_pages, uint8_t* tok_class, void* stream);
 
 /* Sub-token routing and packing (Section 3.3 "Routing mask"; Section 3.4 and
  * Appendix B.1 for the global budget M = N*K; the VLM per-token rule is the
@@ -327,6 +349,23 @@ int32_t stc_pass_host(const stc_shape* shape, const void* k_host, const void* v_
                       float sm_scale, int64_t cap_groups, void* arena, size_t arena_bytes,
                       float* out_host, int64_t* total_groups_host, int32_t* status_host,
                       void* stream);
+
+/* One decode step from HOST memory over a cache that is resident on the device
+ * (the per-step read side: Stage I selection, Section 3.2, then the routed
+ * attention of Section 3.3): copies q from q_host into the arena, runs
+ * stc_quest_select (skipped when token_budget < 0: every page attended) and
+ * stc_decode_attn on `cache` (device pointers: k, kmin, kmax, v_packed, v_mask,
+ * v_offs as left by the write-side calls), and copies out [B][Hq][128] and the
+ * attention call's device status word (STC_OK or STC_ERR_TIMEOUT) to host
+ * buffers.  Everything is enqueued on `stream`; the host outputs are valid after
+ * the caller synchronises it.  q_host / out_host / status_host should be
+ * page-locked.  arena: device memory, 256-byte aligned, at least
+ * stc_decode_step_host_arena_bytes() bytes, owned by the caller, reusable by the
+ * next call on the same stream.  Errors are those of the two calls it chains. */
+int32_t stc_decode_step_host_arena_bytes(const stc_shape* shape, int32_t token_budget, size_t* bytes_host);
+int32_t stc_decode_step_host(const stc_shape* shape, const stc_cache* cache, const void* q_host,
+                             int32_t token_budget, float sm_scale, void* arena, size_t arena_bytes,
+                             float* out_host, int32_t* status_host, void* stream);
 
 #ifdef __cplusplus
 }

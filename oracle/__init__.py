@@ -205,6 +205,20 @@ def select_batch(q, kmin, kmax, token_budget, t_cap, seq_len=None, max_pages=Non
     return (ids, n, sc) if want_scores else (ids, n)
 
 
+def near_ties_batch(q, kmin, kmax, token_budget, t_cap, seq_len=None, rel=1e-6):
+    """i32 [B,Hkv]: pages (other than the k-th itself) whose fp64 bound lies within
+    rel*max(1,|U_k|) of the k-th largest bound of their problem."""
+    B, Hq, _ = q.shape
+    Hkv = kmin.shape[1]
+    counts = np.zeros((B, Hkv), np.int32)
+    sl = None if seq_len is None else np.ascontiguousarray(seq_len, np.int32)
+    lib().stc_o_near_ties_batch(C.c_int32(B), C.c_int32(Hq), C.c_int32(Hkv), C.c_int32(t_cap), _p(sl),
+                                _p(np.ascontiguousarray(q), np.uint16), _p(np.ascontiguousarray(kmin), np.uint16),
+                                _p(np.ascontiguousarray(kmax), np.uint16), C.c_int32(token_budget),
+                                C.c_double(rel), _p(counts))
+    return counts
+
+
 def route_pack_batch(v, scores, cls, S, k_nominal, cap_groups, seq_len=None, min_per_token=1,
                      mode=MODE_GLOBAL, cls_per_head=False):
     """v uint16 [B,Hkv,T,128]; scores f32 [B,Hkv,T,S]; cls uint8 [B,T] / [B,Hkv,T] / None."""
@@ -273,3 +287,20 @@ def query_bias(h_q, w_q, q_len=None):
                            _p(np.ascontiguousarray(h_q), np.uint16), _p(ql),
                            _p(np.ascontiguousarray(w_q), np.uint16), _p(s_q), _p(bias))
     return s_q, bias
+
+
+def pages_to_class(page_ids, n_pages, t_cap, seq_len=None):
+    """Token classes of the paper's own stage order (Section 3.4 / Appendix B.1: the router sees the
+    tokens Stage I retained): uint8 [B,Hkv,T], ROUTED for the valid tokens of the listed pages of each
+    (batch, kv head) problem, DROP elsewhere.  Plain loops."""
+    B, Hkv, _ = page_ids.shape
+    cls = np.full((B, Hkv, t_cap), CLS_DROP, np.uint8)
+    for b in range(B):
+        length = t_cap if seq_len is None else int(seq_len[b])
+        for h in range(Hkv):
+            for i in range(int(n_pages[b, h])):
+                p = int(page_ids[b, h, i])
+                for t in range(p * PAGE, min((p + 1) * PAGE, length)):
+                    if t >= 0:
+                        cls[b, h, t] = CLS_ROUTED
+    return cls

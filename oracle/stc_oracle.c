@@ -442,6 +442,50 @@ void stc_o_select_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const
                               n_pages, scores_out);
 }
 
+/* Near-tie count of the page selection, per problem: with U64[p] = max over the problem's query
+ * heads of the bound accumulated in fp64 (stc_o_bound_f64) and U_k its k-th largest value
+ * (k = min(n_pages, budget / 16)), the number of OTHER pages with |U64[p] - U_k| <=
+ * rel * max(1, |U_k|).  0 when every page or no page is selected.  A reporting aid: these are the
+ * pages whose membership in the selection hangs on the last bits of the fp32 sum. */
+static int f64_desc(const void* a, const void* b) {
+    double x = *(const double*)a, y = *(const double*)b;
+    return x > y ? -1 : (x < y ? 1 : 0);
+}
+
+void stc_o_near_ties_batch(int32_t B, int32_t Hq, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,
+                           const uint16_t* q, const uint16_t* kmin, const uint16_t* kmax,
+                           int32_t token_budget, double rel, int32_t* counts /* [B][Hkv] */) {
+    int32_t p_cap = (t_cap + PAGE - 1) / PAGE;
+    int32_t gq = Hq / Hkv;
+#pragma omp parallel for schedule(static)
+    for (int32_t pr = 0; pr < B * Hkv; ++pr) {
+        int32_t b = pr / Hkv, hk = pr % Hkv;
+        int32_t np = (len_of(seq_len, b, t_cap) + PAGE - 1) / PAGE;
+        int32_t k = token_budget / PAGE < np ? token_budget / PAGE : np;
+        counts[pr] = 0;
+        if (k <= 0 || k >= np) continue;
+        double* u = (double*)malloc(sizeof(double) * (size_t)np * 2);
+        double* sorted = u + np;
+        for (int32_t p = 0; p < np; ++p) {
+            double best = 0.0;
+            for (int32_t h = 0; h < gq; ++h) {
+                double x = stc_o_bound_f64(q + ((size_t)b * Hq + (size_t)hk * gq + h) * D,
+                                           kmin + ((size_t)pr * p_cap + p) * D, kmax + ((size_t)pr * p_cap + p) * D);
+                if (h == 0 || x > best) best = x;
+            }
+            u[p] = best;
+        }
+        memcpy(sorted, u, sizeof(double) * (size_t)np);
+        qsort(sorted, (size_t)np, sizeof(double), f64_desc);
+        double uk = sorted[k - 1];
+        double tol = rel * (fabs(uk) > 1.0 ? fabs(uk) : 1.0);
+        int32_t c = 0;
+        for (int32_t p = 0; p < np; ++p) c += fabs(u[p] - uk) <= tol;
+        counts[pr] = c - 1;
+        free(u);
+    }
+}
+
 /* status [B*Hkv]: 0 ok, -1 budget below one group per token, -2 bad args,
  * -3 capacity overflow.  total [B*Hkv] = groups kept. */
 void stc_o_route_pack_batch(int32_t B, int32_t Hkv, int32_t t_cap, const int32_t* seq_len,

@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window", "stc_pages_to_class", "stc_decode_step_host_arena_bytes", "stc_decode_step_host",
 )
 
 
@@ -75,6 +75,8 @@ def load_library():
                                                 C.c_void_p]
         lib.stc_quest_select_static.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32,
                                                 C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.stc_pages_to_class.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                           C.c_void_p]
         lib.stc_route_pack.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                        C.c_int32, C.c_int32, C.c_int32, C.POINTER(_Cache), C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -96,6 +98,9 @@ def load_library():
         lib.stc_pass_host.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_int64,
                                       C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.stc_decode_step_host_arena_bytes.argtypes = [C.POINTER(_Shape), C.c_int32, C.POINTER(C.c_size_t)]
+        lib.stc_decode_step_host.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32, C.c_float,
+                                             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -227,6 +232,14 @@ def quest_select_static(shape: Shape, cache: Cache, q: torch.Tensor, token_budge
         _ptr(scores, torch.float32, "scores"), _stream()), "stc_quest_select_static")
 
 
+def pages_to_class(shape: Shape, page_ids: torch.Tensor, n_pages: torch.Tensor, tok_class: torch.Tensor) -> None:
+    """tok_class u8 [B,Hkv,T] <- ROUTED for the valid tokens of the listed pages, DROP elsewhere."""
+    cs = shape.c()
+    _check(load_library().stc_pages_to_class(
+        C.byref(cs), _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"),
+        page_ids.shape[-1], _ptr(tok_class, torch.uint8, "tok_class"), _stream()), "stc_pages_to_class")
+
+
 def route_pack(shape: Shape, v: torch.Tensor, scores: torch.Tensor, tok_class: Optional[torch.Tensor],
                k_nominal: int, cache: Cache, total_groups: torch.Tensor, status: torch.Tensor,
                ws: torch.Tensor, min_per_token: int = 1, mode: int = MODE_GLOBAL) -> None:
@@ -343,3 +356,22 @@ def pass_host(shape: Shape, k: torch.Tensor, v: torch.Tensor, scores: torch.Tens
         min_per_token, mode, sm_scale, cap_groups, _ptr(arena, torch.uint8, "arena"), arena.numel(),
         _hptr(out, torch.float32, "out"), _hptr(total_groups, torch.int64, "total_groups"),
         _hptr(status, torch.int32, "status"), _stream()), "stc_pass_host")
+
+
+def decode_step_host_arena_bytes(shape: Shape, token_budget: Optional[int]) -> int:
+    out = C.c_size_t(0)
+    cs = shape.c()
+    _check(load_library().stc_decode_step_host_arena_bytes(
+        C.byref(cs), -1 if token_budget is None else token_budget, C.byref(out)), "stc_decode_step_host_arena_bytes")
+    return int(out.value)
+
+
+def decode_step_host(shape: Shape, cache: Cache, q: torch.Tensor, token_budget: Optional[int], sm_scale: float,
+                     arena: torch.Tensor, out: torch.Tensor, status: torch.Tensor) -> None:
+    """One decode step (page selection + routed attention) on a device-resident cache, query and result in
+    (pinned) host tensors; the results are valid after a stream sync."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_decode_step_host(
+        C.byref(cs), C.byref(cc), _hptr(q, torch.bfloat16, "q"), -1 if token_budget is None else token_budget,
+        sm_scale, _ptr(arena, torch.uint8, "arena"), arena.numel(), _hptr(out, torch.float32, "out"),
+        _hptr(status, torch.int32, "status"), _stream()), "stc_decode_step_host")

@@ -64,6 +64,48 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr) {
     return r;
 }
 
+// ---- mbarrier + 1-D bulk asynchronous copy (the untiled TMA path) ---------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for the phase `parity` of an mbarrier.  False = gave up after limit_ns.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+#pragma unroll 1
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > limit_ns) return false;
+    }
+}
+// 1-D bulk copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned; bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
 // Order-preserving map from fp32 to uint32 (larger float -> larger key); -0 is folded
 // onto +0 (by the addition) so the two compare equal.
 __device__ __forceinline__ uint32_t float_key(float f) {
@@ -75,6 +117,37 @@ __device__ __forceinline__ float key_float(uint32_t k) {
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
+// Inclusive prefix sum over the lanes of a warp.
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+
+// Packed bf16 min / max of two words.
+__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
+    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// Multiprocessor count of the current device (queried per call: cheap next to a launch, and
+// right on every device of a multi-GPU process).
+inline cudaError_t device_sm_count(int* n) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(n, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess && *n <= 0) e = cudaErrorInvalidDevice;
+    return e;
+}
+
 // ---- internal launchers (one per source file) -------------------------------
 cudaError_t launch_page_meta(const Geom& g, const void* k, void* kmin, void* kmax, int page_begin,
                              int page_end, cudaStream_t st);
@@ -83,6 +156,9 @@ size_t select_ws_bytes(const Geom& g);
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
                                 int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
                                 int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st);
+
+cudaError_t launch_pages_to_class(const Geom& g, const int32_t* page_ids, const int32_t* n_pages,
+                                  int max_pages, uint8_t* tok_class, cudaStream_t st);
 
 size_t route_ws_bytes(const Geom& g);
 cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,

@@ -12,14 +12,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kPagesPerCta = kThreads / 16;
 
-__device__ __forceinline__ uint32_t bmin2(uint32_t a, uint32_t b) {
-    __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
-    return *reinterpret_cast<uint32_t*>(&r);
-}
-__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b) {
-    __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
-    return *reinterpret_cast<uint32_t*>(&r);
-}
 
 __global__ void __launch_bounds__(kThreads)
 page_meta_kernel(const uint4* __restrict__ k, uint4* __restrict__ kmin, uint4* __restrict__ kmax,

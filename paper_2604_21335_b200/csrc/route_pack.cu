@@ -75,14 +75,6 @@ __device__ __forceinline__ uint32_t pass_himask(int pass) {
     return pass == 0 ? 0u : (pass == 1 ? 0xFFE00000u : 0xFFFFFC00u);
 }
 
-__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, v, d);
-        if (lane >= d) v += o;
-    }
-    return v;
-}
 
 // Block-wide exclusive scan of one value per thread (kThreads threads).
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w /*[kWarps]*/, uint32_t* total) {

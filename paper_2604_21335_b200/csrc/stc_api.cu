@@ -111,6 +111,18 @@ int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, 
                                        static_cast<cudaStream_t>(stream)));
 }
 
+int32_t stc_pages_to_class(const stc_shape* shape, const int32_t* page_ids, const int32_t* n_pages,
+                           int32_t max_pages, uint8_t* tok_class, void* stream) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (max_pages < 0) return STC_ERR_INVALID_ARG;
+    if (empty(g)) return STC_OK;
+    if (!tok_class || (max_pages > 0 && (!page_ids || !n_pages))) return STC_ERR_INVALID_ARG;
+    return cuda_rc(launch_pages_to_class(g, page_ids, n_pages, max_pages, tok_class,
+                                         static_cast<cudaStream_t>(stream)));
+}
+
 namespace {
 int32_t route_pack_phases(const stc_shape* shape, const void* v, const float* scores,
                           const uint8_t* tok_class, int64_t class_head_stride, int32_t k_nominal,
@@ -354,6 +366,69 @@ int32_t stc_pass_host(const stc_shape* shape, const void* k_host, const void* v_
         e = cudaMemcpyAsync(total_groups_host, a.total, (size_t)g.problems * 8, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(status_host, a.status, (size_t)g.problems * 4, cudaMemcpyDeviceToHost, st);
+    return cuda_rc(e);
+}
+
+
+namespace {
+struct StepArena { char *q, *ids, *npages, *out, *ws; size_t ws_bytes, total_bytes; int max_pages; };
+StepArena carve_step_arena(const Geom& g, int token_budget, void* base) {
+    StepArena a;
+    char* p = static_cast<char*>(base);
+    size_t o = 0;
+    auto take = [&](size_t bytes) { char* r = p + o; o += up256(bytes); return r; };
+    a.max_pages = token_budget < 0 ? g.P : (token_budget / kPage < g.P ? token_budget / kPage : g.P);
+    if (a.max_pages < 1) a.max_pages = 1;
+    a.q = take((size_t)g.B * g.Hq * kRowBytes);
+    a.ids = take((size_t)g.problems * a.max_pages * 4);
+    a.npages = take((size_t)g.problems * 4);
+    a.out = take((size_t)g.B * g.Hq * kHeadDim * 4);
+    // selection and attention keep separate workspaces: the attention status word must survive
+    const size_t ws_sel = up256(select_ws_bytes(g)), ws_att = up256(attn_ws_bytes(g, a.max_pages));
+    a.ws_bytes = ws_att;
+    a.ws = take(ws_att);
+    take(ws_sel);
+    a.total_bytes = o;
+    return a;
+}
+}  // namespace
+
+int32_t stc_decode_step_host_arena_bytes(const stc_shape* shape, int32_t token_budget, size_t* bytes_host) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (!bytes_host) return STC_ERR_INVALID_ARG;
+    *bytes_host = empty(g) ? 0 : carve_step_arena(g, token_budget, nullptr).total_bytes;
+    return STC_OK;
+}
+
+int32_t stc_decode_step_host(const stc_shape* shape, const stc_cache* cache, const void* q_host,
+                             int32_t token_budget, float sm_scale, void* arena, size_t arena_bytes,
+                             float* out_host, int32_t* status_host, void* stream) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (!cache || !q_host || !out_host || !status_host) return STC_ERR_INVALID_ARG;
+    if (empty(g)) return STC_OK;
+    const StepArena a = carve_step_arena(g, token_budget, arena);
+    rc = check_ws(arena, arena_bytes, a.total_bytes);
+    if (rc != STC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(a.q, q_host, (size_t)g.B * g.Hq * kRowBytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return STC_ERR_CUDA;
+    const int32_t* ids = nullptr;
+    if (token_budget >= 0) {
+        rc = stc_quest_select(shape, cache, a.q, token_budget, a.max_pages, reinterpret_cast<int32_t*>(a.ids),
+                              reinterpret_cast<int32_t*>(a.npages), nullptr, a.ws + a.ws_bytes,
+                              up256(select_ws_bytes(g)), stream);
+        if (rc != STC_OK) return rc;
+        ids = reinterpret_cast<const int32_t*>(a.ids);
+    }
+    rc = stc_decode_attn(shape, cache, a.q, ids, reinterpret_cast<const int32_t*>(a.npages), a.max_pages,
+                         sm_scale, reinterpret_cast<float*>(a.out), nullptr, a.ws, a.ws_bytes, stream);
+    if (rc != STC_OK) return rc;
+    cudaError_t e = cudaMemcpyAsync(out_host, a.out, (size_t)g.B * g.Hq * kHeadDim * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(status_host, a.ws, 4, cudaMemcpyDeviceToHost, st);
     return cuda_rc(e);
 }
 

@@ -242,43 +242,6 @@ def test_cfg3_full_size_whole_batch():
     assert o["page_ids"] is None and (o["total"] == 128 * 8 + 144 * 3).all()
 
 
-@pytest.mark.parametrize("name,samples", [("cfg1", [(0, 0), (0, 13), (0, 31)]),
-                                          ("cfg2", [(0, 0), (5, 2), (7, 3)]),
-                                          ("cfg4", [(0, 0), (9, 5)])])
-def test_full_size_sampled_problems(name, samples):
-    """At the benchmarked sizes: whole pass on the GPU, sampled problems on the checker."""
-    w = W.get(name)
-    d = W.make_inputs(w, DEV)
-    g = H.gpu_pipeline(w, d)
-    S = w.n_groups
-    # properties that hold at any size
-    cnt = torch.zeros_like(g["cache"].v_mask, dtype=torch.int32)
-    for j in range(S):
-        cnt += (g["cache"].v_mask.int() >> j) & 1
-    assert (cnt.sum(-1) == w.t_cache * w.k_nominal).all() and cnt.min() >= 1
-    assert (g["total"] == w.t_cache * w.k_nominal).all() and (g["status"] == 0).all()
-    offs = g["cache"].v_offs.long()
-    assert torch.equal(offs[..., 1:] - offs[..., :-1], cnt.long())
-    ids = g["page_ids"]
-    assert (ids[..., 1:] > ids[..., :-1]).all() and (g["n_pages"] == w.token_budget // 16).all()
-    for b, hk in samples:
-        w1, d1 = _problem_slice(w, d, b, hk)
-        o = H.oracle_pipeline(w1, d1)
-        g1 = dict(cache=P.Cache(kmin=g["cache"].kmin[b:b + 1, hk:hk + 1].contiguous(),
-                                kmax=g["cache"].kmax[b:b + 1, hk:hk + 1].contiguous(),
-                                v_mask=g["cache"].v_mask[b:b + 1, hk:hk + 1].contiguous(),
-                                v_offs=g["cache"].v_offs[b:b + 1, hk:hk + 1].contiguous(),
-                                v_packed=g["cache"].v_packed[b:b + 1, hk:hk + 1].contiguous()),
-                  total=g["total"][b:b + 1, hk:hk + 1], status=g["status"][b:b + 1, hk:hk + 1],
-                  page_ids=g["page_ids"][b:b + 1, hk:hk + 1], n_pages=g["n_pages"][b:b + 1, hk:hk + 1],
-                  u=g["u"][b:b + 1, hk:hk + 1],
-                  out=g["out"][b:b + 1, hk * w.gq:(hk + 1) * w.gq],
-                  lse=g["lse"][b:b + 1, hk * w.gq:(hk + 1) * w.gq])
-        H.assert_bit_exact_write_side(w1, g1, o)
-        H.assert_bit_exact_selection(g1, o)
-        H.assert_attention_close(g1, o)
-
-
 @pytest.mark.parametrize("name,S,T", [("cfg0", 8, 1300), ("cfg2", 16, 16 * 70 + 3)])
 def test_many_medium_problems_span_the_ranges_of_the_selection_ctas(name, S, T):
     """Hundreds of problems, each a few 256-token units long (too long for the one-CTA kernel):

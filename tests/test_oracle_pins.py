@@ -508,3 +508,39 @@ def test_select_recent_window_against_brute_force():
     # no window = the plain rule
     u = g.standard_normal(64).astype(np.float32)
     np.testing.assert_array_equal(O.select(u, 256, 0), O.select(u, 256))
+
+
+def test_pages_to_class_hand_example():
+    # two problems, 40-token rows; problem 0 lists pages 2 and 0 of a 35-token sequence (page 2 is partial),
+    # problem 1 lists nothing
+    ids = np.array([[[2, 0, 1], [1, 1, 1]]], np.int32)
+    n = np.array([[2, 0]], np.int32)
+    cls = O.pages_to_class(ids, n, 40, np.array([35], np.int32))
+    want0 = np.zeros(40, np.uint8); want0[0:16] = 1; want0[32:35] = 1
+    assert cls.shape == (1, 2, 40)
+    np.testing.assert_array_equal(cls[0, 0], want0)
+    assert (cls[0, 1] == 0).all()
+
+
+def test_near_tie_count_on_a_constructed_row_of_bounds():
+    # One channel carries the whole bound: q[0] = 1, kmin[p][0] = kmax[p][0] = value_p, so U[p] = value_p exactly
+    # (values are exact in bf16).  k = 3 pages: sorted values 9, 8, [5], 5, 5, 4.984375(bf16 step 2^-6 below 5), 1.
+    bf = lambda x: (np.array([x], np.float32).view(np.uint32) >> 16).astype(np.uint16)[0]
+    vals = [5.0, 9.0, 1.0, 5.0, 8.0, 4.96875, 5.0]
+    P_ = len(vals)
+    kmin = np.zeros((1, 1, P_, 128), np.uint16); kmax = np.zeros((1, 1, P_, 128), np.uint16)
+    for p, x in enumerate(vals):
+        assert np.float32(x) == O.bits_to_f32(np.array([bf(x)], np.uint16))[0]
+        kmin[0, 0, p, 0] = kmax[0, 0, p, 0] = bf(x)
+    q = np.zeros((1, 1, 128), np.uint16); q[0, 0, 0] = bf(1.0)
+    T = 16 * P_
+    assert O.near_ties_batch(q, kmin, kmax, 3 * 16, T)[0, 0] == 2            # the two other pages equal to 5
+    assert O.near_ties_batch(q, kmin, kmax, 3 * 16, T, rel=0.01)[0, 0] == 3  # 4.96875 is within 1 % of 5
+    assert O.near_ties_batch(q, kmin, kmax, 1 * 16, T)[0, 0] == 0            # 9 stands alone
+    assert O.near_ties_batch(q, kmin, kmax, 2 * 16, T)[0, 0] == 0            # so does 8
+    assert O.near_ties_batch(q, kmin, kmax, 7 * 16, T)[0, 0] == 0            # everything selected: nothing to decide
+    assert O.near_ties_batch(q, kmin, kmax, 0, T)[0, 0] == 0
+    # a second head whose bound is larger on one page takes over there (max over the group's heads)
+    q2 = np.zeros((1, 2, 128), np.uint16); q2[0, 0, 0] = bf(1.0); q2[0, 1, 1] = bf(1.0)
+    kmin[0, 0, 2, 1] = kmax[0, 0, 2, 1] = bf(5.0)                           # page 2: head 1 sees 5 instead of 1
+    assert O.near_ties_batch(q2, kmin, kmax, 3 * 16, T)[0, 0] == 3
