@@ -448,6 +448,8 @@ __device__ __noinline__ float exact_page_score(const uint4* __restrict__ kmin_ro
 // sum_c max(q kmin, q kmax); the same products on absolute values give sum_c |term|, whose
 // largest value over the problem scales the error margin of the filter.
 constexpr int kFilterMinGq = 2;               // single-head problems stay on the fp32 pipes
+constexpr int kFilterMinPages = 4096;         // pages per problem from which the filtered scan is the faster one
+constexpr int kFilterMinPagesSplit = 1024;    // ... with more than four query heads per KV head
 constexpr int kFDepth = 2;                                       // tiles in flight per warp
 constexpr int kFCtasPerSm = 1;
 constexpr uint32_t kFTileBytes = 16u * 512u;                     // 8 KiB per tile: kmax rows | kmin rows
@@ -1107,10 +1109,12 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
     int sms = 0;
     e = device_sm_count(&sms);
     if (e != cudaSuccess) return e;
-    // Several query heads per KV head and no score output: the tensor-core scan filters, the
-    // declared-order fp32 bound settles the pages near the threshold.  Otherwise every page gets
-    // the declared-order bound on the fp32 pipes.
-    const bool filter = scores_opt == nullptr && g.Gq >= kFilterMinGq;
+    // Several query heads per KV head, long rows of pages and no score output: the tensor-core scan
+    // filters, the declared-order fp32 bound settles the pages near the threshold (one CTA per SM, a
+    // heavier per-problem selection: it pays once a problem's scan outweighs that).  Otherwise every
+    // page gets the declared-order bound on the fp32 pipes.
+    const bool filter = scores_opt == nullptr &&
+                        ((g.Gq >= kFilterMinGq && g.P >= kFilterMinPages) || (g.Gq > 4 && g.P >= kFilterMinPagesSplit));
     const int pages_per_unit = filter ? kFUnitPages : kWarps * (g.Gq > 4 ? 1 : 2);
     const int units_per_problem = (g.P + pages_per_unit - 1) / pages_per_unit;
     const long long total_units = (long long)units_per_problem * g.problems;

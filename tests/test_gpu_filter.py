@@ -56,33 +56,33 @@ def select_both_ways(w, d, seq=None, budget=None, n_recent=0, q_index=0, want_ws
 
 @pytest.mark.parametrize("gq", [2, 3, 4, 5, 7, 8])
 def test_filtered_selection_matches_the_checker(gq):
-    w = W.shrink(W.get("cfg4"), batch=3, n_q_heads=2 * gq, n_kv_heads=2, t_cache=16 * 1234 + 7, token_budget=16 * 150)
+    w = W.shrink(W.get("cfg4"), batch=3, n_q_heads=2 * gq, n_kv_heads=2, t_cache=16 * 4234 + 7, token_budget=16 * 150)
     d = W.make_inputs(w, DEV, n_queries=2)
     for qi in range(2):
         select_both_ways(w, d, seq=[w.t_cache, 16 * 517 + 1, 16 * 128], q_index=qi)
 
 
-@pytest.mark.parametrize("budget", [16, 48, 16 * 700, 16 * 1233])
+@pytest.mark.parametrize("budget", [16, 48, 16 * 700, 16 * 4233])
 def test_budget_extremes(budget):
-    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=8, n_kv_heads=2, t_cache=16 * 1234 + 7)
+    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=8, n_kv_heads=2, t_cache=16 * 4234 + 7)
     d = W.make_inputs(w, DEV)
     select_both_ways(w, d, budget=budget)
 
 
 def test_exact_ties_between_duplicated_pages_go_to_the_lower_page():
-    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=8, n_kv_heads=2, t_cache=16 * 512, token_budget=16 * 61)
+    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=8, n_kv_heads=2, t_cache=16 * 4512, token_budget=16 * 61)
     d = W.make_inputs(w, DEV)
-    k = d["k"].view(1, 2, 512, 16, 128)
+    k = d["k"].view(1, 2, 4512, 16, 128)
     k[:, :, 1::2] = k[:, :, 0::2].clone()                  # every page has an identical twin
     r = select_both_ways(w, d)
     assert H.near_tie_pages(r["u_o"][0, 0], 61) >= 1
 
 
 def test_every_page_identical_takes_the_exact_fallback():
-    # 3000 identical pages: all of them lie inside the margin, far more than the list of pages to settle holds
-    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=8, n_kv_heads=2, t_cache=16 * 3000, token_budget=16 * 100)
+    # 5000 identical pages: all of them lie inside the margin, far more than the list of pages to settle holds
+    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=8, n_kv_heads=2, t_cache=16 * 5000, token_budget=16 * 100)
     d = W.make_inputs(w, DEV)
-    k = d["k"].view(1, 2, 3000, 16, 128)
+    k = d["k"].view(1, 2, 5000, 16, 128)
     k[:] = k[:, :, :1].clone()
     r = select_both_ways(w, d)
     assert (r["n_o"] == 100).all()
@@ -91,11 +91,11 @@ def test_every_page_identical_takes_the_exact_fallback():
 def test_a_crowd_of_near_ties_around_the_threshold():
     # pages 200..1199 are copies of one page with the lowest mantissa bit of ONE key element flipped here and
     # there: their bounds differ by a few ulps, hundreds of them straddle the threshold
-    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=4, n_kv_heads=1, t_cache=16 * 2000, token_budget=16 * 700)
+    w = W.shrink(W.get("cfg4"), batch=1, n_q_heads=4, n_kv_heads=1, t_cache=16 * 4200, token_budget=16 * 700)
     d = W.make_inputs(w, DEV)
-    k = d["k"].view(1, 1, 2000, 16, 128)
+    k = d["k"].view(1, 1, 4200, 16, 128)
     k[:, :, 200:1200] = k[:, :, 200:201].clone()
-    kb = d["k"].view(torch.int16).view(1, 1, 2000, 16, 128)
+    kb = d["k"].view(torch.int16).view(1, 1, 4200, 16, 128)
     g = torch.Generator(device="cpu"); g.manual_seed(5)
     for p in range(200, 1200):
         t, c = int(torch.randint(0, 16, (1,), generator=g)), int(torch.randint(0, 128, (1,), generator=g))
@@ -105,9 +105,9 @@ def test_a_crowd_of_near_ties_around_the_threshold():
 
 @pytest.mark.parametrize("n_recent", [1, 4, 40])
 def test_local_window_with_the_filtered_scan(n_recent):
-    w = W.shrink(W.get("cfg2"), batch=2, t_cache=16 * 300 + 9, token_budget=16 * 30)
+    w = W.shrink(W.get("cfg2"), batch=2, t_cache=16 * 1300 + 9, token_budget=16 * 30)     # Gq = 7
     d = W.make_inputs(w, DEV)
-    select_both_ways(w, d, seq=[16 * 300 + 9, 16 * 37 + 2], n_recent=n_recent)
+    select_both_ways(w, d, seq=[16 * 1300 + 9, 16 * 37 + 2], n_recent=n_recent)
 
 
 def test_rows_too_long_to_stage_in_shared_memory():
@@ -117,11 +117,12 @@ def test_rows_too_long_to_stage_in_shared_memory():
 
 
 def test_many_short_problems_and_empty_sequences():
-    w = W.shrink(W.get("cfg2"), batch=50, n_q_heads=14, n_kv_heads=2, t_cache=16 * 40 + 5, token_budget=16 * 9)
+    # capacity of 1100 pages per sequence (Gq = 7), most sequences far shorter
+    w = W.shrink(W.get("cfg2"), batch=50, n_q_heads=14, n_kv_heads=2, t_cache=16 * 1100 + 5, token_budget=16 * 9)
     d = W.make_inputs(w, DEV)
     g0 = torch.Generator(device="cpu"); g0.manual_seed(3)
-    seq = torch.randint(0, w.t_cache + 1, (50,), generator=g0).tolist()
-    seq[0] = 0; seq[1] = 1; seq[2] = w.t_cache; seq[3] = 16 * 9; seq[4] = 16 * 9 + 1
+    seq = torch.randint(0, 16 * 60, (50,), generator=g0).tolist()
+    seq[0] = 0; seq[1] = 1; seq[2] = w.t_cache; seq[3] = 16 * 9; seq[4] = 16 * 9 + 1; seq[5] = 16 * 700 + 3
     select_both_ways(w, d, seq=seq)
 
 
@@ -130,7 +131,7 @@ def test_the_margin_of_the_filter_has_room_to_spare():
     words per problem -- arrival counters [problems], largest sum|term| [problems], two key bounds -- padded
     to 256 bytes, then f32 [problems][P]) against the declared-order scores: the difference must stay below
     an eighth of the margin the kernel allows itself."""
-    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=16, n_kv_heads=2, t_cache=16 * 4000, token_budget=16 * 200)
+    w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=16, n_kv_heads=2, t_cache=16 * 4100, token_budget=16 * 200)
     d = W.make_inputs(w, DEV)
     r = select_both_ways(w, d, want_ws=True)
     problems, Pn = 4, r["shape"].n_pages

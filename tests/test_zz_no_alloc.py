@@ -89,9 +89,10 @@ def test_static_scratch_holds_the_scores_when_the_caller_passes_none():
     """Without a score tensor the fp32 page scores live in the built-in array: the second call
     starts with the first query's scores still there and must not be influenced by them."""
     dev = "cuda"
-    # several CTAs per problem (1800 pages), Gq = 4 and Gq = 1, ragged lengths
-    for hq, hkv in ((8, 2), (3, 3)):
-        w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=hq, n_kv_heads=hkv, t_cache=16 * 1800 + 11,
+    # several CTAs per problem, ragged lengths: Gq = 4 with 4300 pages (the tensor-core scan, whose approximate
+    # scores and per-problem words live in the array) and Gq = 1 with 1800 pages (the fp32 scan)
+    for hq, hkv, pages in ((8, 2, 4300), (3, 3, 1800)):
+        w = W.shrink(W.get("cfg4"), batch=2, n_q_heads=hq, n_kv_heads=hkv, t_cache=16 * pages + 11,
                      token_budget=16 * 130)
         d = W.make_inputs(w, dev, n_queries=3)
         seq = torch.tensor([w.t_cache, 16 * 977 + 2], dtype=torch.int32, device=dev)
