@@ -23,6 +23,8 @@
 // PER_TOKEN mode skips the histogram passes (the mask is local to a token).
 // HBM traffic: scores 4x (3 passes + mask, from L2 when they fit; 1x in PER_TOKEN
 // mode), kept part of V once in and once out.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace stc {
@@ -264,6 +266,11 @@ __device__ __forceinline__ uint32_t budget_of(uint64_t n_routed, int k_nominal, 
 
 // ---- bounded cross-CTA hand-off -------------------------------------------------
 constexpr uint64_t kWaitNs = 2000000000ull;   // a wait that lasts this long gives up and reports a time-out
+// Launch parameters of the selection kernel that only the library's own tests change (see
+// stc_test_route_select_knobs at the end of this file): the first histogram pass to run and the
+// limit of a hand-off wait.
+std::atomic<int> g_first_pass{0};
+std::atomic<unsigned long long> g_wait_ns{kWaitNs};
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
     uint64_t t;
@@ -283,7 +290,7 @@ __device__ __forceinline__ void st_release(uint32_t* p, uint32_t v) {
 // s_bc = {ok, flags, prefix, krem}.  False (for the whole CTA) after a time-out or when
 // another CTA has already given up.
 __device__ __forceinline__ bool wait_done(const uint32_t* state, uint32_t need, uint32_t* s_bc,
-                                          uint32_t* abort_word) {
+                                          uint32_t* abort_word, uint64_t wait_ns) {
     __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t ok = 1;
@@ -291,7 +298,7 @@ __device__ __forceinline__ bool wait_done(const uint32_t* state, uint32_t need, 
             const uint64_t t0 = globaltimer_ns();
             while (ld_acquire(state + ST_DONE) < need) {
                 __nanosleep(100);
-                if (globaltimer_ns() - t0 > kWaitNs || ld_acquire(abort_word) != 0u) { ok = 0; break; }
+                if (globaltimer_ns() - t0 > wait_ns || ld_acquire(abort_word) != 0u) { ok = 0; break; }
             }
         }
         if (!ok) atomicExch(abort_word, 1u);
@@ -316,7 +323,8 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
                     int k_nominal, int min_per_token, int mode, uint32_t* __restrict__ state_all,
                     uint32_t* __restrict__ hist_all, uint32_t* __restrict__ abort_word,
                     uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
-                    uint32_t* __restrict__ unit_sums, long long total_units) {
+                    uint32_t* __restrict__ unit_sums, long long total_units, int first_pass,
+                    unsigned long long wait_ns) {
     constexpr int kBatch = 32 / S;               // tokens in flight per thread (32 score registers)
     __shared__ uint32_t shist[kBins];
     __shared__ uint32_t s_w[kWarps];
@@ -331,7 +339,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
     const int n_pass = mode == STC_MODE_GLOBAL ? 3 : 0;
 
 #pragma unroll 1
-    for (int pass = 0; pass < n_pass; ++pass) {
+    for (int pass = first_pass; pass < n_pass; ++pass) {
         const uint32_t himask = pass_himask(pass);
         const int dshift = pass_shift(pass);
         const uint32_t dmask = pass == 2 ? 1023u : 2047u;
@@ -360,7 +368,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             load_batch(u0);                              // in flight while the digit of the previous pass arrives
             uint32_t prefix = 0, krem_in = 0;
             if (pass > 0) {
-                if (!wait_done(state, (uint32_t)pass, s_bc, abort_word)) return;
+                if (!wait_done(state, (uint32_t)pass, s_bc, abort_word, wait_ns)) return;
                 if (s_bc[1] != 0u) continue;             // nothing to select / budget error: resolved in pass 0
                 prefix = s_bc[2];
                 krem_in = s_bc[3];
@@ -460,7 +468,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
         load_batch(u0);                                  // in flight while the last digit arrives
         uint32_t tau = 0, flags = 0;
         if (mode == STC_MODE_GLOBAL) {
-            if (!wait_done(state_all + (size_t)problem * ST_WORDS, 3u, s_bc, abort_word)) return;
+            if (!wait_done(state_all + (size_t)problem * ST_WORDS, 3u, s_bc, abort_word, wait_ns)) return;
             flags = s_bc[1];
             tau = s_bc[2];
         }
@@ -748,8 +756,10 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
     int Hkv = g.Hkv, T = g.T;
     uint32_t *state = w.state, *hist = w.hist, *abort_word = w.abort_word, *unit_sums = w.unit_sums;
     uint16_t* tie = w.tie;
+    int first_pass = g_first_pass.load();
+    unsigned long long wait_ns = g_wait_ns.load();
     void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token, &mode,
-                    &state, &hist, &abort_word, &v_mask, &tie, &unit_sums, &total_units};
+                    &state, &hist, &abort_word, &v_mask, &tie, &unit_sums, &total_units, &first_pass, &wait_ns};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_select_kernel<S>), dim3(grid),
                                        dim3(kThreads), args, 0, st);
 }
@@ -801,4 +811,18 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
     return cudaGetLastError();
 }
 
+void set_route_select_knobs(int first_pass, unsigned long long wait_ns) {
+    g_first_pass.store(first_pass < 0 || first_pass > 3 ? 0 : first_pass);
+    g_wait_ns.store(wait_ns ? wait_ns : kWaitNs);
+}
+
 }  // namespace stc
+
+// Test hook, not part of the public interface (not declared in stc.h): makes the cooperative
+// selection kernel start at histogram pass `first_pass` (0 = normal) and bound its hand-off waits by
+// wait_ns (0 = the default of two seconds).  With first_pass = 3 on a freshly cleared workspace no
+// CTA ever publishes a digit, so every wait runs into its limit and the give-up path (abort word,
+// orderly return, STC_ERR_TIMEOUT from the packing kernel) executes without anything hanging.
+extern "C" void stc_test_route_select_knobs(int32_t first_pass, uint64_t wait_ns) {
+    stc::set_route_select_knobs(first_pass, wait_ns);
+}
