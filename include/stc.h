@@ -294,6 +294,29 @@ int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const 
                           const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
                           void* stream);
 
+/* Routing of the pages completed during decoding (Section 3.4: the budget is global over the
+ * retained tokens, M = N*K in Appendix B.1, and the query region stays uncompressed; the paper
+ * does not say when a generated token leaves the query region -- reading taken: while its
+ * 16-token page is still open).  For every sequence b with len = shape->seq_len[b], each complete
+ * page p with first_page[b] <= p < len/16 -- stored at full width by stc_append_tokens -- is
+ * routed ON ITS OWN: its 16 tokens join the routed set, the budget grows by 16*k_nominal groups
+ * and they are allotted among the page's (token, group) pairs by the rule of stc_route_pack
+ * (STC_MODE_GLOBAL with floor min_per_token: each token's first maximum, then the best
+ * 16*k_nominal - 16 of the page's other pairs, ties to the lower flat index; STC_MODE_PER_TOKEN:
+ * every token's k_nominal best groups).  The kept groups are compacted in place, the tokens of
+ * the still open page stay at full width and move down behind them; v_mask, v_offs[first..len]
+ * and total_groups are updated.  The result does not depend on whether pages are routed one
+ * call at a time or several at once, and the routed tokens always hold exactly N*k_nominal
+ * groups.
+ *   scores      f32 [B][Hkv][t_cap][S], rows of the completed pages are read
+ *   first_page  device i32 [B]: first page not yet routed
+ * At most 8 pages per sequence and call.  status i32 [B][Hkv]: STC_OK; STC_ERR_INVALID_ARG
+ * (more than 8 completed pages, or the range is not stored at full width) and STC_ERR_BUDGET
+ * (k_nominal = 0 with floor 1) leave the problem untouched.  Needs no workspace. */
+int32_t stc_route_new_pages(const stc_shape* shape, const stc_cache* cache, const float* scores,
+                            const int32_t* first_page, int32_t k_nominal, int32_t min_per_token,
+                            int32_t mode, int64_t* total_groups, int32_t* status, void* stream);
+
 /* Routed decode attention (Section 3.3, attention equation): per query head h
  * with KV head h / (Hq/Hkv) and R = the valid tokens of the listed pages,
  *     s_t = sm_scale * q_h.k_t,  p = softmax over R of s,

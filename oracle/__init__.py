@@ -50,6 +50,7 @@ def lib():
         _lib.stc_o_select.restype = C.c_int32
         _lib.stc_o_route.restype = C.c_int32
         _lib.stc_o_pack.restype = C.c_int64
+        _lib.stc_o_route_new_pages.restype = C.c_int64
         _lib.stc_o_kv_fraction.restype = C.c_double
         _lib.stc_o_max_threads.restype = C.c_int32
     return _lib
@@ -140,6 +141,20 @@ def pack(v: np.ndarray, mask: np.ndarray, S: int, cap_groups: int):
     n = lib().stc_o_pack(_p(np.ascontiguousarray(v), np.uint16), _p(np.ascontiguousarray(mask), np.uint16),
                          C.c_int32(T), C.c_int32(S), C.c_int64(cap_groups), _p(offs), _p(packed))
     return int(n), offs, packed
+
+
+def route_new_pages(scores, length, S, first_page, k_nominal, mask, offs, packed, min_per_token=1,
+                    mode=MODE_GLOBAL):
+    """In place on one problem: the complete pages from first_page on (stored at full width) are routed
+    page by page, the open page's tokens move down.  scores f32 [T,S], mask u16 [T], offs u32 [T+1],
+    packed u16 [cap,128/S].  Returns the new total (or -1 / -2, nothing changed)."""
+    assert scores.dtype == np.float32 and mask.dtype == np.uint16 and offs.dtype == np.uint32
+    assert packed.dtype == np.uint16
+    for a in (scores, mask, offs, packed):
+        assert a.flags["C_CONTIGUOUS"]
+    return int(lib().stc_o_route_new_pages(_p(scores), C.c_int32(length), C.c_int32(S), C.c_int32(first_page),
+                                           C.c_int32(k_nominal), C.c_int32(min_per_token), C.c_int32(mode),
+                                           _p(mask), _p(offs), _p(packed)))
 
 
 def attend_packed(q, k, packed, mask, offs, length, S, page_ids, scale):

@@ -245,6 +245,54 @@ int32_t stc_o_route(const float* scores, const uint8_t* cls, int32_t len, int32_
 }
 
 /* ------------------------------------------------------------------------
+ * Routing of pages completed during decoding (Section 3.4: global budget over the retained
+ * tokens, M = N*K in Appendix B.1, query-region tokens uncompressed; the paper does not say
+ * when a generated token leaves the query region -- reading taken: while its 16-token page is
+ * still open; when the page completes, its 16 tokens join the routed set and the budget grows
+ * by 16*K groups, which are allotted among the page's own (token, group) pairs by the rule of
+ * stc_o_route, because the dropped groups of older tokens no longer exist in a packed store).
+ *
+ * One problem, in place.  Tokens first_page*16 .. len-1 are stored at full width (mask all
+ * ones) behind the earlier tokens' groups.  Every complete page p, first_page <= p < len/16,
+ * is routed on its own with scores [len][S] (rows of those pages are read); the tokens of the
+ * still open page stay at full width and move down behind the compacted pages.  mask [len],
+ * offs [len+1], packed [cap][128/S] are updated.  Returns the new total, -1 when the budget is
+ * below one group per token with min_per_token = 1 (nothing changed), -2 on bad arguments or
+ * when the range is not stored at full width (nothing changed).
+ * ---------------------------------------------------------------------- */
+int64_t stc_o_route_new_pages(const float* scores, int32_t len, int32_t S, int32_t first_page,
+                              int32_t k_nominal, int32_t min_per_token, int32_t mode,
+                              uint16_t* mask, uint32_t* offs, uint16_t* packed) {
+    int g = D / S;
+    int32_t t0 = first_page * PAGE;
+    int32_t n_pages = len / PAGE - first_page;
+    if (first_page < 0 || S < 1 || S > 16 || k_nominal < 0 || k_nominal > S) return -2;
+    if (n_pages <= 0 || t0 >= len) return (int64_t)offs[len];
+    for (int32_t t = t0; t < len; ++t)
+        if (mask[t] != (uint16_t)((1u << S) - 1u) || offs[t + 1] - offs[t] != (uint32_t)S) return -2;
+    if (mode == MODE_GLOBAL && min_per_token && k_nominal < 1) return -1;
+    /* the full-width values of the range, read out before anything is overwritten */
+    int32_t n_tok = len - t0;
+    uint16_t* full = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)n_tok * D);
+    memcpy(full, packed + (size_t)offs[t0] * g, sizeof(uint16_t) * (size_t)n_tok * D);
+    for (int32_t p = 0; p < n_pages; ++p)
+        stc_o_route(scores + (size_t)(t0 + p * PAGE) * S, NULL, PAGE, S, k_nominal, min_per_token, mode,
+                    mask + t0 + p * PAGE);
+    int64_t n = offs[t0];
+    for (int32_t t = t0; t < len; ++t) {
+        offs[t] = (uint32_t)n;
+        for (int j = 0; j < S; ++j) {
+            if (!((mask[t] >> j) & 1u)) continue;
+            memcpy(packed + (size_t)n * g, full + (size_t)(t - t0) * D + (size_t)j * g, sizeof(uint16_t) * (size_t)g);
+            ++n;
+        }
+    }
+    offs[len] = (uint32_t)n;
+    free(full);
+    return n;
+}
+
+/* ------------------------------------------------------------------------
  * Packing: walk the tokens in order; offs[t] is the number of groups kept
  * before token t (offs[len] = total); the kept groups of a token are stored
  * in ascending group order, each group_dim = 128/S bf16 values.

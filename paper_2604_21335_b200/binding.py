@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window", "stc_pages_to_class", "stc_decode_step_host_arena_bytes", "stc_decode_step_host",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window", "stc_pages_to_class", "stc_route_new_pages", "stc_decode_step_host_arena_bytes", "stc_decode_step_host",
 )
 
 
@@ -86,6 +86,8 @@ def load_library():
                                         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_append_tokens.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.stc_route_new_pages.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_int32,
+                                            C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_query_bias.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.stc_router_logits.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
@@ -283,6 +285,17 @@ def append_tokens(shape: Shape, cache: Cache, v: torch.Tensor, old_len: torch.Te
         C.byref(cs), C.byref(cc), _ptr(v, torch.bfloat16, "v"), _ptr(old_len, torch.int32, "old_len"), max_new,
         _ptr(total_groups, torch.int64, "total_groups"), _ptr(status, torch.int32, "status"), _stream()),
         "stc_append_tokens")
+
+
+def route_new_pages(shape: Shape, cache: Cache, scores: torch.Tensor, first_page: torch.Tensor, k_nominal: int,
+                    total_groups: torch.Tensor, status: torch.Tensor, min_per_token: int = 1,
+                    mode: int = MODE_GLOBAL) -> None:
+    """Routes, page by page, the complete pages from first_page[b] on (stored at full width by append_tokens)."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_route_new_pages(
+        C.byref(cs), C.byref(cc), _ptr(scores, torch.float32, "scores"), _ptr(first_page, torch.int32, "first_page"),
+        k_nominal, min_per_token, mode, _ptr(total_groups, torch.int64, "total_groups"),
+        _ptr(status, torch.int32, "status"), _stream()), "stc_route_new_pages")
 
 
 def router_logits(shape: Shape, h: torch.Tensor, w: torch.Tensor, scores: torch.Tensor, status_word: torch.Tensor,

@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libstc.so"
-SOURCES = ["stc_api.cu", "page_meta.cu", "quest_select.cu", "quest_select_static.cu", "page_class.cu", "route_pack.cu", "append.cu", "router.cu", "query_bias.cu", "decode_attn.cu"]
+SOURCES = ["stc_api.cu", "page_meta.cu", "quest_select.cu", "quest_select_static.cu", "page_class.cu", "route_pack.cu", "append.cu", "route_pages.cu", "router.cu", "query_bias.cu", "decode_attn.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC",

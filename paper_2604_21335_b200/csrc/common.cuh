@@ -173,6 +173,12 @@ cudaError_t launch_append(const Geom& g, const void* k, void* kmin, void* kmax, 
                           uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups, int32_t* status,
                           cudaStream_t st);
 
+int route_new_pages_max();
+cudaError_t launch_route_new_pages(const Geom& g, const float* scores, const int32_t* first_page, int k_nominal,
+                                   int min_per_token, int mode, void* v_packed, uint16_t* v_mask,
+                                   uint32_t* v_offs, int64_t cap_groups, int64_t* total_groups, int32_t* status,
+                                   cudaStream_t st);
+
 cudaError_t launch_router_logits(const Geom& g, const void* h, const void* w, const float* bias, int d_model,
                                  float* scores, int32_t* status, cudaStream_t st);
 

@@ -217,6 +217,24 @@ int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const 
                                  static_cast<cudaStream_t>(stream)));
 }
 
+int32_t stc_route_new_pages(const stc_shape* shape, const stc_cache* cache, const float* scores,
+                            const int32_t* first_page, int32_t k_nominal, int32_t min_per_token,
+                            int32_t mode, int64_t* total_groups, int32_t* status, void* stream) {
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (!cache || k_nominal < 0 || k_nominal > g.S || (min_per_token != 0 && min_per_token != 1) ||
+        (mode != STC_MODE_GLOBAL && mode != STC_MODE_PER_TOKEN))
+        return STC_ERR_INVALID_ARG;
+    if (empty(g)) return STC_OK;
+    if (!cache->v_packed || !cache->v_mask || !cache->v_offs || cache->cap_groups < 0 || !scores || !first_page ||
+        !total_groups || !status)
+        return STC_ERR_INVALID_ARG;
+    return cuda_rc(launch_route_new_pages(g, scores, first_page, k_nominal, min_per_token, mode, cache->v_packed,
+                                          cache->v_mask, cache->v_offs, cache->cap_groups, total_groups, status,
+                                          static_cast<cudaStream_t>(stream)));
+}
+
 int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const void* q,
                         const int32_t* page_ids, const int32_t* n_pages, int32_t max_pages,
                         float sm_scale, float* out, float* lse_opt, void* ws, size_t ws_bytes,

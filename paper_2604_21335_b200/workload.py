@@ -83,6 +83,8 @@ CONFIGS: Dict[str, Workload] = {
     # batch axis (the library treats every (batch, kv head) problem independently, so a stack
     # of layers is just a larger batch) -- amortises the per-call latency of the small configs
     "cfg1x32": Workload("cfg1x32", 32, 32, 32, 32768, 8, 4, 2048, "vnorm", seed=0x5C7C0011),
+    # cfg2 for all 28 layers of the Qwen2.5-7B-shaped model in one call (7 query heads per KV head, S = 16)
+    "cfg2x28": Workload("cfg2x28", 8 * 28, 28, 4, 32768, 16, 4, 4096, "normal", seed=0x5C7C0012),
     # long-context GQA sweep base point (budget / k_nominal overridden per point)
     "cfg4": Workload("cfg4", 16, 32, 8, 131072, 8, 4, 4096, "normal", seed=0x5C7C0004),
 }

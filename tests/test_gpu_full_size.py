@@ -132,3 +132,34 @@ def test_cfg4_every_problem_and_every_sweep_point_at_full_context(cfg4, keep):
             worst[bud][0] = max(worst[bud][0], ma); worst[bud][1] = max(worst[bud][1], mr)
         del x, kmin, kmax, r, o
     print(f"cfg4 keep {keep}: worst attention error per budget {worst}")
+
+
+@pytest.mark.parametrize("name,chunk", [("cfg1x32", 4), ("cfg2x28", 28)])
+def test_all_layers_in_one_call(name, chunk):
+    """The layer-stacked workloads (every layer's cache along the batch axis, one call per step for the
+    whole model): the whole pass on the GPU at full size, every problem against the checker, `chunk`
+    sequences at a time."""
+    w = W.get(name)
+    d = W.make_inputs(w, DEV)
+    cap = w.t_cache * w.k_nominal
+    g = H.gpu_pipeline(w, d, cap_groups=cap)
+    assert (g["status"] == 0).all() and (g["total"] == cap).all()
+    assert (g["n_pages"] == w.token_budget // 16).all()
+    wc = W.shrink(w, batch=chunk)
+    worst = [0.0, 0.0]
+    for b0 in range(0, w.batch, chunk):
+        sl = slice(b0, b0 + chunk)
+        dc = dict(k=d["k"][sl], v=d["v"][sl], q=d["q"][:, sl], scores=d["scores"][sl], tok_class=None,
+                  seq_len=d["seq_len"][sl])
+        o = H.oracle_pipeline(wc, dc, cap_groups=cap)
+        c = g["cache"]
+        gc = dict(cache=P.Cache(kmin=c.kmin[sl], kmax=c.kmax[sl], v_mask=c.v_mask[sl], v_offs=c.v_offs[sl],
+                                v_packed=c.v_packed[sl]),
+                  total=g["total"][sl], status=g["status"][sl], page_ids=g["page_ids"][sl],
+                  n_pages=g["n_pages"][sl], u=g["u"][sl], out=g["out"][sl], lse=g["lse"][sl])
+        H.assert_bit_exact_write_side(wc, gc, o)
+        H.assert_bit_exact_selection(gc, o)
+        ma, mr = H.assert_attention_close(gc, o)
+        worst = [max(worst[0], ma), max(worst[1], mr)]
+        del o
+    print(f"{name}: worst attention error {worst}")

@@ -96,6 +96,30 @@ def test_routing_modes(kn, mpt, mode):
     full_parity(w, min_per_token=mpt, mode=mode)
 
 
+# The paper's own (S, K) settings: fixed per-token top-K for the VLMs (S4K1, S8K2, S16K4: Section 3.5,
+# Appendix C.2) and the global budget for the LLMs (S8K7, S8K6, S16K14, S16K12: Table 3, Appendix C.1).
+PAPER_GRID = [(4, 1, 1), (8, 2, 1), (16, 4, 1), (8, 7, 0), (8, 6, 0), (16, 14, 0), (16, 12, 0)]
+
+
+@pytest.mark.parametrize("S,K,mode", PAPER_GRID)
+def test_paper_grid_of_groups_and_budgets(S, K, mode):
+    # long enough for the cooperative selection kernel (several 256-token units per problem), ragged lengths
+    w = W.shrink(W.get("cfg0"), batch=2, n_q_heads=4, n_kv_heads=4, t_cache=16 * 330 + 5, token_budget=16 * 40,
+                 n_groups=S, k_nominal=K)
+    d, g, o, _ = full_parity(w, seq_len=[w.t_cache, 16 * 97 + 9], mode=mode)
+    cnt = np.vectorize(lambda x: bin(int(x)).count("1"))(o["mask"])
+    for b, L in enumerate(o["seq_len"]):
+        if mode == 1:
+            assert (cnt[b, :, :L] == K).all()                       # every token keeps exactly K groups
+        else:
+            assert (cnt[b, :, :L].sum(-1) == L * K).all() and cnt[b, :, :L].min() >= 1
+    # the VLM-shaped cache (text tokens at full width) with the per-token rule
+    if mode == 1:
+        w3 = W.shrink(W.get("cfg3"), batch=2, n_q_heads=4, n_kv_heads=4, n_groups=S, k_nominal=K)
+        d3, g3, o3, _ = full_parity(w3, mode=1)
+        assert (o3["total"] == 128 * S + 144 * K).all()
+
+
 @pytest.mark.parametrize("mode", [0, 1])
 def test_route_mask_then_pack_values_equals_route_pack(mode):
     w = W.shrink(W.get("cfg2"), batch=2, t_cache=2500, k_nominal=3)

@@ -544,3 +544,88 @@ def test_near_tie_count_on_a_constructed_row_of_bounds():
     q2 = np.zeros((1, 2, 128), np.uint16); q2[0, 0, 0] = bf(1.0); q2[0, 1, 1] = bf(1.0)
     kmin[0, 0, 2, 1] = kmax[0, 0, 2, 1] = bf(5.0)                           # page 2: head 1 sees 5 instead of 1
     assert O.near_ties_batch(q2, kmin, kmax, 3 * 16, T)[0, 0] == 3
+
+
+def _popcounts(mask):
+    return np.vectorize(lambda x: bin(int(x)).count("1"))(mask)
+
+
+@pytest.mark.parametrize("S,K,mpt,mode", [(8, 4, 1, 0), (8, 7, 1, 0), (16, 4, 1, 0), (4, 1, 1, 1), (8, 2, 0, 0), (8, 8, 1, 0)])
+def test_routing_of_pages_completed_during_decoding(S, K, mpt, mode):
+    """A decode loop on the checker: a routed prefix, then tokens appended at full width; complete
+    pages are routed as they close.  Pinned by (a) the running budget: the routed tokens always hold
+    exactly N*K groups (Appendix B.1), the open page S per token; (b) the data: unpacking the store gives
+    V with the dropped groups zeroed, for every token, after every step (the in-place compaction moved
+    the right bytes); (c) a second construction that never compacts in place: the final masks packed
+    from the dense values in one sequential walk; (d) the page rule itself: each completed page's
+    masks are those of the (exhaustively pinned) routing rule applied to that page alone; (e) routing the
+    closed pages one call at a time or several at once gives the same store."""
+    rng = np.random.default_rng(100 + S + K)
+    g = 128 // S
+    T0, T1 = 16 * 3 + 5, 16 * 9 + 11                      # prefix ends inside a page; 6 pages close during the loop
+    v = rng.integers(1, 2 ** 16, size=(T1, 128), dtype=np.uint16)
+    sc = np.round(rng.standard_normal((T1, S)).astype(np.float32) * 4) / 4    # ties
+    cap = T1 * S
+    # prefix: routed up to the last complete page, its open page at full width
+    cls = np.ones(T0, np.uint8); cls[16 * 3:] = O.CLS_FULL
+    rc, m0 = O.route(sc[:T0], cls, S, K, mpt, mode)
+    assert rc == 0
+    mask = np.zeros(T1, np.uint16); mask[:T0] = m0
+    total, offs0, packed = O.pack(v[:T0], mask[:T0], S, cap)
+    offs = np.zeros(T1 + 1, np.uint32); offs[:T0 + 1] = offs0
+
+    def check(length, first_open_page):
+        routed = first_open_page * 16
+        cnt = _popcounts(mask[:length])
+        if mode == 1:
+            assert (cnt[:routed] == K).all()
+        else:
+            assert cnt[:routed].sum() == routed * K                      # M = N*K at every step
+            if mpt:
+                assert cnt[:routed].min() >= 1
+        assert (cnt[routed:length] == S).all()
+        assert (np.diff(offs[:length + 1].astype(np.int64)) == cnt).all()
+        for t in range(length):                                          # unpack == V with dropped groups removed
+            o = int(offs[t])
+            for j in range(S):
+                if (mask[t] >> j) & 1:
+                    np.testing.assert_array_equal(packed[o], v[t, j * g:(j + 1) * g]); o += 1
+
+    length, first_open = T0, 3
+    snapshots = {}
+    for t in range(T0, T1):                                              # append one token at full width
+        mask[t] = (1 << S) - 1
+        for j in range(S):
+            packed[int(offs[t]) + j] = v[t, j * g:(j + 1) * g]
+        offs[t + 1] = offs[t] + S
+        length = t + 1
+        if length % 16 == 0:
+            if length // 16 in (5, 6):                                   # let two pages pile up, route them together
+                if length // 16 == 5:
+                    continue
+            new_total = O.route_new_pages(sc, length, S, first_open, K, mask, offs, packed, mpt, mode)
+            assert new_total == int(offs[length])
+            first_open = length // 16
+            check(length, first_open)
+            snapshots[length] = (mask[:length].copy(), packed[:new_total].copy())
+    check(length, first_open)
+    # (c) + (d): the same final state built without any in-place step
+    want = np.zeros(T1, np.uint16); want[:16 * 3] = m0[:16 * 3]
+    for p in range(3, T1 // 16):
+        rc, mp_ = O.route(sc[16 * p:16 * p + 16], None, S, K, mpt, mode)
+        assert rc == 0
+        want[16 * p:16 * p + 16] = mp_
+    want[(T1 // 16) * 16:] = (1 << S) - 1
+    np.testing.assert_array_equal(mask, want)
+    total2, offs2, packed2 = O.pack(v, want, S, cap)
+    np.testing.assert_array_equal(offs, offs2)
+    np.testing.assert_array_equal(packed[:total2], packed2[:total2])
+    # refusals leave everything as it was
+    before = (mask.copy(), offs.copy(), packed.copy())
+    if K < S:
+        assert O.route_new_pages(sc, T1, S, 2, K, mask, offs, packed, mpt, mode) == -2  # page 2 is not at full width
+    if mode == 0 and mpt == 1:
+        m2 = mask.copy(); m2[T1 - 11:] = (1 << S) - 1
+        assert O.route_new_pages(sc, T1 - 11 + 16, S, T1 // 16, 0, m2, offs.copy(), packed.copy(), 1, 0) in (-1, -2)
+    for a, b in zip(before, (mask, offs, packed)):
+        np.testing.assert_array_equal(a, b)
