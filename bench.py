@@ -411,6 +411,39 @@ def run_gpu(args, r: D.Rank):
     for c in copies:
         assert int(c.status.abs().sum()) == 0
 
+    # ---- the write side from hidden states: router logits (tcgen05 GEMM) -> masks -> packed store ----
+    write_from_hidden = None
+    if not args.no_router and (Hkv * S <= 256 or (Hkv * S) % 256 == 0):
+        c0 = copies[0]
+        dm = D_MODEL.get(w.name.split("x")[0], 4096)
+        gen = torch.Generator(device=dev); gen.manual_seed(w.seed ^ 0x707)
+        hs = torch.empty(B, T, dm, dtype=torch.bfloat16, device=dev)
+        for b in range(B):
+            hs[b] = torch.randn(T, dm, generator=gen, device=dev).to(torch.bfloat16)
+        wt = (torch.randn(Hkv * S, dm, generator=gen, device=dev) / dm ** 0.5).to(torch.bfloat16)
+        sc2 = torch.empty(B, Hkv, T, S, dtype=torch.float32, device=dev)
+        st_word = torch.zeros(1, dtype=torch.int32, device=dev)
+        cache2 = P.Cache.allocate(c0.shape, c0.d["k"], T * S if w.n_text else c0.cap)
+        tot2, stat2 = torch.zeros_like(c0.total), torch.zeros_like(c0.status)
+
+        def from_hidden():
+            P.router_logits(c0.shape, hs, wt, sc2, st_word)
+            P.route_mask(c0.shape, sc2, c0.d["tok_class"], w.k_nominal, cache2, c0.ws_r)
+            P.pack_values(c0.shape, c0.d["v"], cache2, tot2, stat2, c0.ws_r)
+
+        t_all = timed(graphed(from_hidden), max(2, min(20, int(budget_ms / max(sum(per_call_ms[1:3]) * 2, 1e-3)))))
+        t_rt = timed(graphed(lambda: P.router_logits(c0.shape, hs, wt, sc2, st_word)),
+                     max(2, min(20, int(budget_ms / max(per_call_ms[1], 1e-3)))))
+        torch.cuda.synchronize()
+        assert int(st_word[0]) == 0 and int(stat2.abs().sum()) == 0
+        rt_bytes = B * T * dm * 2 + Hkv * S * dm * 2 + B * T * Hkv * S * 4
+        write_from_hidden = {"us": round(t_all * 1e3, 2), "router_logits_us": round(t_rt * 1e3, 2),
+                             "router_logits_GBps": round(rt_bytes / (t_rt * 1e-3) / 1e9, 1),
+                             "router_logits_TFLOPs": round(2.0 * B * T * Hkv * S * dm / (t_rt * 1e-3) / 1e12, 1),
+                             "d_model": dm,
+                             "calls": "stc_router_logits -> stc_route_mask -> stc_pack_values (synthetic router weights)"}
+        del hs, sc2, cache2
+
     # ---- the CPU checker on a sample of problems: timed baseline, parity check, near-tie count ----
     probs = sample_problems(w, args.cpu_problems)
     cpu_baseline = checked = None
@@ -573,6 +606,7 @@ def run_gpu(args, r: D.Rank):
                       "GBps": round(pass_bytes / (pass_ms * 1e-3) / 1e9, 1),
                       "streams": "one" if args.serial else "two (page metadata | routing + packing, joined before the decode step)"},
         "e2e_full_pass": e2e_pass,
+        "write_side_from_hidden": write_from_hidden,
         "tokens_heads_per_s": {"context": round(B * Hq * T * r.world / (ms_per_step * 1e-3)),
                                "attended": round(sel_tokens * w.gq * r.world / (ms_per_step * 1e-3))},
     }
@@ -704,6 +738,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-e2e-pass", action="store_true", help="skip the whole pass from host buffers")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-router", action="store_true", help="skip the write side measured from hidden states")
     ap.add_argument("--serial", action="store_true", help="the write side of the full pass on one stream")
     ap.add_argument("--only", default=None, choices=["router"], help="time one extra kernel instead of the step")
     args = ap.parse_args()

@@ -51,7 +51,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    subprocess.check_call([nvcc, "-shared", "-o", str(tmp), *objs, "-lcudart"])
+    subprocess.check_call([nvcc, "-shared", "-o", str(tmp), *objs, "-lcudart", "-ldl"])
     os.replace(tmp, LIB)
     return LIB
 

@@ -1,5 +1,7 @@
 // C-ABI of libstc: host-side argument validation and dispatch.  Nothing here
 // allocates device memory; every launch goes to the caller's stream.
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 using namespace stc;
@@ -32,6 +34,12 @@ int32_t check_ws(const void* ws, size_t have, size_t need) {
 }
 
 int32_t cuda_rc(cudaError_t e) { return e == cudaSuccess ? STC_OK : STC_ERR_CUDA; }
+
+// NVTX range around the host side of a call (what it enqueues shows under it in a timeline).
+struct Range {
+    explicit Range(const char* name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
 
 }  // namespace
 
@@ -74,6 +82,7 @@ int32_t stc_workspace_bytes(const stc_shape* shape, int32_t op, int64_t arg, siz
 
 int32_t stc_build_page_meta(const stc_shape* shape, const stc_cache* cache, int32_t page_begin,
                             int32_t page_end, void* stream) {
+    Range nvtx_range("stc_build_page_meta");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -96,6 +105,7 @@ int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, 
                                 int32_t token_budget, int32_t n_recent_pages, int32_t max_pages,
                                 int32_t* page_ids, int32_t* n_pages, float* scores_opt, void* ws,
                                 size_t ws_bytes, void* stream) {
+    Range nvtx_range("stc_quest_select_window");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -113,6 +123,7 @@ int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, 
 
 int32_t stc_pages_to_class(const stc_shape* shape, const int32_t* page_ids, const int32_t* n_pages,
                            int32_t max_pages, uint8_t* tok_class, void* stream) {
+    Range nvtx_range("stc_pages_to_class");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -155,6 +166,7 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
                        int32_t min_per_token, int32_t mode, const stc_cache* out,
                        int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes,
                        void* stream) {
+    Range nvtx_range("stc_route_pack");
     return route_pack_phases(shape, v, scores, tok_class, class_head_stride, k_nominal, min_per_token, mode,
                              out, total_groups, status, ws, ws_bytes, 3, stream);
 }
@@ -162,18 +174,21 @@ int32_t stc_route_pack(const stc_shape* shape, const void* v, const float* score
 int32_t stc_route_mask(const stc_shape* shape, const float* scores, const uint8_t* tok_class,
                        int64_t class_head_stride, int32_t k_nominal, int32_t min_per_token, int32_t mode,
                        const stc_cache* out, void* ws, size_t ws_bytes, void* stream) {
+    Range nvtx_range("stc_route_mask");
     return route_pack_phases(shape, nullptr, scores, tok_class, class_head_stride, k_nominal, min_per_token,
                              mode, out, nullptr, nullptr, ws, ws_bytes, 1, stream);
 }
 
 int32_t stc_pack_values(const stc_shape* shape, const void* v, int32_t mode, const stc_cache* out,
                         int64_t* total_groups, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+    Range nvtx_range("stc_pack_values");
     return route_pack_phases(shape, v, nullptr, nullptr, 0, 0, 0, mode, out, total_groups, status, ws,
                              ws_bytes, 2, stream);
 }
 
 int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, const float* bias_opt,
                           int32_t d_model, float* scores, int32_t* status_word, void* stream) {
+    Range nvtx_range("stc_router_logits");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -191,6 +206,7 @@ int32_t stc_router_logits(const stc_shape* shape, const void* h, const void* w, 
 
 int32_t stc_query_bias(int32_t batch, int32_t q_cap, int32_t d_model, int32_t n_logits, const void* h_q,
                        const int32_t* q_len_opt, const void* w_q, float* s_q, float* bias, void* stream) {
+    Range nvtx_range("stc_query_bias");
     if (batch < 0 || q_cap < 0 || d_model <= 0 || n_logits < 0 || batch > 65535) return STC_ERR_INVALID_ARG;
     if (d_model % 8 != 0) return STC_ERR_UNSUPPORTED;
     if (batch == 0) return STC_OK;
@@ -204,6 +220,7 @@ int32_t stc_query_bias(int32_t batch, int32_t q_cap, int32_t d_model, int32_t n_
 int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const void* v,
                           const int32_t* old_len, int32_t max_new, int64_t* total_groups, int32_t* status,
                           void* stream) {
+    Range nvtx_range("stc_append_tokens");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -220,6 +237,7 @@ int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const 
 int32_t stc_route_new_pages(const stc_shape* shape, const stc_cache* cache, const float* scores,
                             const int32_t* first_page, int32_t k_nominal, int32_t min_per_token,
                             int32_t mode, int64_t* total_groups, int32_t* status, void* stream) {
+    Range nvtx_range("stc_route_new_pages");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -239,6 +257,7 @@ int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const vo
                         const int32_t* page_ids, const int32_t* n_pages, int32_t max_pages,
                         float sm_scale, float* out, float* lse_opt, void* ws, size_t ws_bytes,
                         void* stream) {
+    Range nvtx_range("stc_decode_attn");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -336,6 +355,7 @@ int32_t stc_pass_host(const stc_shape* shape, const void* k_host, const void* v_
                       float sm_scale, int64_t cap_groups, void* arena, size_t arena_bytes,
                       float* out_host, int64_t* total_groups_host, int32_t* status_host,
                       void* stream) {
+    Range nvtx_range("stc_pass_host");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
@@ -423,6 +443,7 @@ int32_t stc_decode_step_host_arena_bytes(const stc_shape* shape, int32_t token_b
 int32_t stc_decode_step_host(const stc_shape* shape, const stc_cache* cache, const void* q_host,
                              int32_t token_budget, float sm_scale, void* arena, size_t arena_bytes,
                              float* out_host, int32_t* status_host, void* stream) {
+    Range nvtx_range("stc_decode_step_host");
     Geom g;
     int32_t rc = make_geom(shape, &g);
     if (rc != STC_OK) return rc;
