@@ -577,7 +577,9 @@ def run_gpu(args, r: D.Rank):
     step_calls = {n: per_call_ms[names.index(n)] for n in ("quest_select", "decode_attn") if ab[n]}
     dom = max(step_calls, key=step_calls.get)
     traffic = TRAFFIC_NOTE.get((w.name, w.batch, w.token_budget, w.k_nominal, dom))
-    roof = {"bound": "hbm", "kernel": KERNEL_OF[dom] + (f"<{w.gq}>" if dom == "quest_select" else ""),
+    sel_kernel = ("quest_filter_kernel" if (w.gq >= 2 and w.n_pages >= 4096) or (w.gq > 4 and w.n_pages >= 1024)
+                  else "quest_select_kernel") + f"<{w.gq}>"      # the library's own choice of scan, restated
+    roof = {"bound": "hbm", "kernel": sel_kernel if dom == "quest_select" else KERNEL_OF[dom],
             "achieved": per_kernel[dom]["GBps"], "peak": peak, "unit": UNIT,
             "frac": round(per_kernel[dom]["GBps"] / peak, 4), "peak_source": peak_src + " copy bandwidth",
             "traffic": traffic}
@@ -616,7 +618,7 @@ def run_gpu(args, r: D.Rank):
     print(json.dumps(line), flush=True)
 
 
-KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kernel",
+KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kernel",   # (or quest_filter_kernel, see below)
              "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel",
              "route_mask": "route_select_kernel"}
 
@@ -624,6 +626,10 @@ KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kern
 # kernel from the committed ncu captures under profiles/, keyed by (workload, batch, budget, keep, call);
 # absent = no capture of the kernel as it stands.
 TRAFFIC_NOTE: dict = {
+    # quest_filter_kernel<4>: dram__bytes_read 134.62 MB + dram__bytes_write 4.01 MB per launch at batch 4
+    # (profiles/ncu_full_select_attn_cfg4_batch4.md), scaled by 4 to the 16 sequences of the full workload (the
+    # traffic is the metadata scan plus the score array, both proportional to the number of problems)
+    ("cfg4", 16, 4096, 4, "quest_select"): 4 * (134.62e6 + 4.01e6),
 }
 
 
