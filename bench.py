@@ -201,7 +201,7 @@ def sample_problems(w: W.Workload, n: int):
 def workload_string(w: W.Workload) -> str:
     return (f"{w.name}: B{w.batch} Hq{w.n_q_heads} Hkv{w.n_kv_heads} T{w.t_cache} S{w.n_groups} "
             f"keep{w.k_nominal} budget{w.token_budget}, one decode step per step "
-            "(stc_quest_select + stc_decode_attn over the resident compressed cache)")
+            "(stc_quest_select + stc_decode_attn over the resident compressed cache)")     # = stc_decode_step
 
 
 L2_BYTES = 126 << 20
@@ -284,6 +284,10 @@ def run_gpu(args, r: D.Rank):
 
     def read_step(j):
         c = copy_of(j)
+        if ids[j] is not None and not args.two_calls:
+            # stc_decode_step = stc_quest_select + stc_decode_attn as one call
+            P.decode_step(c.shape, c.cache, c.qs[j], w.token_budget, ids[j], npg[j], SM_SCALE, out, ws_s, ws_a)
+            return
         if ids[j] is not None:
             P.quest_select(c.shape, c.cache, c.qs[j], w.token_budget, ids[j], npg[j], ws_s)
         P.decode_attn(c.shape, c.cache, c.qs[j], ids[j], npg[j], SM_SCALE, out, ws_a)
@@ -744,6 +748,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-e2e-pass", action="store_true", help="skip the whole pass from host buffers")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--two-calls", action="store_true",
+                    help="time the decode step as stc_quest_select + stc_decode_attn instead of stc_decode_step")
     ap.add_argument("--no-router", action="store_true", help="skip the write side measured from hidden states")
     ap.add_argument("--serial", action="store_true", help="the write side of the full pass on one stream")
     ap.add_argument("--only", default=None, choices=["router"], help="time one extra kernel instead of the step")

@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "stc_status_string", "stc_version", "stc_workspace_bytes", "stc_build_page_meta",
     "stc_quest_select", "stc_route_pack", "stc_decode_attn", "stc_cache_bytes",
-    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window", "stc_pages_to_class", "stc_route_new_pages", "stc_decode_step_host_arena_bytes", "stc_decode_step_host",
+    "stc_pass_host_arena_bytes", "stc_pass_host", "stc_quest_select_static", "stc_route_mask", "stc_pack_values", "stc_append_tokens", "stc_router_logits", "stc_query_bias", "stc_quest_select_window", "stc_pages_to_class", "stc_route_new_pages", "stc_decode_step", "stc_decode_step_host_arena_bytes", "stc_decode_step_host",
 )
 
 
@@ -95,6 +95,9 @@ def load_library():
         lib.stc_decode_attn.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                         C.c_void_p]
+        lib.stc_decode_step.argtypes = [C.POINTER(_Shape), C.POINTER(_Cache), C.c_void_p, C.c_int32, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_size_t, C.c_void_p, C.c_size_t, C.c_void_p]
         lib.stc_cache_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         lib.stc_pass_host_arena_bytes.argtypes = [C.POINTER(_Shape), C.c_int64, C.c_int32, C.POINTER(C.c_size_t)]
         lib.stc_pass_host.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -328,6 +331,18 @@ def decode_attn(shape: Shape, cache: Cache, q: torch.Tensor, page_ids: Optional[
         _ptr(n_pages, torch.int32, "n_pages"), max_pages, sm_scale, _ptr(out, torch.float32, "out"),
         _ptr(lse, torch.float32, "lse"), _ptr(ws, torch.uint8, "ws"), ws.numel(), _stream()),
         "stc_decode_attn")
+
+
+def decode_step(shape: Shape, cache: Cache, q: torch.Tensor, token_budget: int, page_ids: torch.Tensor,
+                n_pages: torch.Tensor, sm_scale: float, out: torch.Tensor, ws_select: torch.Tensor,
+                ws_attn: torch.Tensor, lse: Optional[torch.Tensor] = None) -> None:
+    """quest_select + decode_attn as one call (both workspaces cleared up front, the kernels back to back)."""
+    cs, cc = shape.c(), cache.c()
+    _check(load_library().stc_decode_step(
+        C.byref(cs), C.byref(cc), _ptr(q, torch.bfloat16, "q"), token_budget, page_ids.shape[-1],
+        _ptr(page_ids, torch.int32, "page_ids"), _ptr(n_pages, torch.int32, "n_pages"), sm_scale,
+        _ptr(out, torch.float32, "out"), _ptr(lse, torch.float32, "lse"), _ptr(ws_select, torch.uint8, "ws_select"),
+        ws_select.numel(), _ptr(ws_attn, torch.uint8, "ws_attn"), ws_attn.numel(), _stream()), "stc_decode_step")
 
 
 def cache_bytes(n_tokens_retained: int, n_groups_kept: int, n_groups: int):

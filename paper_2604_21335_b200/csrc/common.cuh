@@ -148,6 +148,11 @@ inline cudaError_t device_sm_count(int* n) {
     return e;
 }
 
+// Launch options of the internal launchers.
+enum : unsigned {
+    kLaunchNoClear = 1u    // the caller has already cleared the call's status / counter words on the stream
+};
+
 // ---- internal launchers (one per source file) -------------------------------
 cudaError_t launch_page_meta(const Geom& g, const void* k, void* kmin, void* kmax, int page_begin,
                              int page_end, cudaStream_t st);
@@ -155,7 +160,8 @@ cudaError_t launch_page_meta(const Geom& g, const void* k, void* kmin, void* kma
 size_t select_ws_bytes(const Geom& g);
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
                                 int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
-                                int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st);
+                                int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st, unsigned flags = 0);
+cudaError_t clear_quest_select_ws(const Geom& g, void* ws, cudaStream_t st);
 
 cudaError_t launch_pages_to_class(const Geom& g, const int32_t* page_ids, const int32_t* n_pages,
                                   int max_pages, uint8_t* tok_class, cudaStream_t st);
@@ -192,6 +198,7 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
                                const uint16_t* v_mask, const uint32_t* v_offs, int64_t cap_groups,
                                const void* q, const int32_t* page_ids, const int32_t* n_pages,
                                int max_pages, float sm_scale, float* out, float* lse, void* ws,
-                               cudaStream_t st);
+                               cudaStream_t st, unsigned flags = 0);
+cudaError_t clear_decode_attn_ws(const Geom& g, void* ws, cudaStream_t st);
 
 }  // namespace stc

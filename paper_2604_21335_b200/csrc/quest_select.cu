@@ -1094,9 +1094,13 @@ size_t select_ws_bytes(const Geom& g) {
     return 256 + counters_bytes(g) + (size_t)g.problems * g.P * sizeof(float);
 }
 
+cudaError_t clear_quest_select_ws(const Geom& g, void* ws, cudaStream_t st) {
+    return cudaMemsetAsync(ws, 0, 256 + (size_t)g.problems * 16, st);
+}
+
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,
                                 int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
-                                int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st) {
+                                int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st, unsigned flags) {
     if (g.problems == 0) return cudaSuccess;
     // workspace: status word (its own 256 bytes), the per-problem words, the page scores
     int32_t* status = static_cast<int32_t*>(ws);
@@ -1104,7 +1108,8 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
     ProblemStats stats{counters, counters + g.problems, counters + 2 * (size_t)g.problems, counters + 3 * (size_t)g.problems};
     float* scores = scores_opt ? scores_opt
                                : reinterpret_cast<float*>(static_cast<char*>(ws) + 256 + counters_bytes(g));
-    cudaError_t e = cudaMemsetAsync(ws, 0, 256 + (size_t)g.problems * 16, st);
+    cudaError_t e = cudaSuccess;
+    if (!(flags & kLaunchNoClear)) e = clear_quest_select_ws(g, ws, st);
     if (e != cudaSuccess) return e;
     int sms = 0;
     e = device_sm_count(&sms);

@@ -278,6 +278,48 @@ int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const vo
                                       out, lse_opt, ws, static_cast<cudaStream_t>(stream)));
 }
 
+int32_t stc_decode_step(const stc_shape* shape, const stc_cache* cache, const void* q, int32_t token_budget,
+                        int32_t max_pages, int32_t* page_ids, int32_t* n_pages, float sm_scale, float* out,
+                        float* lse_opt, void* ws_select, size_t ws_select_bytes, void* ws_attn,
+                        size_t ws_attn_bytes, void* stream) {
+    Range nvtx_range("stc_decode_step");
+    Geom g;
+    int32_t rc = make_geom(shape, &g);
+    if (rc != STC_OK) return rc;
+    if (!cache || token_budget < 0 || max_pages < 0 || !(sm_scale == sm_scale)) return STC_ERR_INVALID_ARG;
+    if (g.problems == 0) return STC_OK;
+    if (!q || !out || !page_ids || !n_pages) return STC_ERR_INVALID_ARG;
+    if (g.T == 0 || max_pages < 1) {              // nothing to select or attend: the two plain calls handle it
+        rc = stc_quest_select(shape, cache, q, token_budget, max_pages, page_ids, n_pages, nullptr, ws_select,
+                              ws_select_bytes, stream);
+        if (rc != STC_OK) return rc;
+        return stc_decode_attn(shape, cache, q, page_ids, n_pages, max_pages, sm_scale, out, lse_opt, ws_attn,
+                               ws_attn_bytes, stream);
+    }
+    if (!cache->kmin || !cache->kmax || !cache->k || !cache->v_packed || !cache->v_mask || !cache->v_offs ||
+        cache->cap_groups < 0)
+        return STC_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v_packed)) & 15u) != 0)
+        return STC_ERR_INVALID_ARG;
+    const int want = token_budget / kPage < g.P ? token_budget / kPage : g.P;
+    if (max_pages < want || max_pages > g.P) return STC_ERR_INVALID_ARG;
+    rc = check_ws(ws_select, ws_select_bytes, select_ws_bytes(g));
+    if (rc == STC_OK) rc = check_ws(ws_attn, ws_attn_bytes, attn_ws_bytes(g, max_pages));
+    if (rc != STC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // both workspaces are cleared first, so that nothing stands between the two kernels
+    cudaError_t e = clear_quest_select_ws(g, ws_select, st);
+    if (e == cudaSuccess) e = clear_decode_attn_ws(g, ws_attn, st);
+    if (e == cudaSuccess)
+        e = launch_quest_select(g, cache->kmin, cache->kmax, q, token_budget, 0, max_pages, page_ids, n_pages,
+                                nullptr, ws_select, st, kLaunchNoClear);
+    if (e == cudaSuccess)
+        e = launch_decode_attn(g, cache->k, cache->v_packed, cache->v_mask, cache->v_offs, cache->cap_groups, q,
+                               page_ids, n_pages, max_pages, sm_scale, out, lse_opt, ws_attn, st,
+                               kLaunchNoClear);
+    return cuda_rc(e);
+}
+
 int32_t stc_cache_bytes(int64_t n_tokens_retained, int64_t n_groups_kept, int32_t n_groups,
                         int64_t* kv_bytes_host, int64_t* index_bytes_host) {
     if (n_tokens_retained < 0 || n_groups_kept < 0 || !kv_bytes_host) return STC_ERR_INVALID_ARG;
@@ -455,16 +497,14 @@ int32_t stc_decode_step_host(const stc_shape* shape, const stc_cache* cache, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(a.q, q_host, (size_t)g.B * g.Hq * kRowBytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return STC_ERR_CUDA;
-    const int32_t* ids = nullptr;
     if (token_budget >= 0) {
-        rc = stc_quest_select(shape, cache, a.q, token_budget, a.max_pages, reinterpret_cast<int32_t*>(a.ids),
-                              reinterpret_cast<int32_t*>(a.npages), nullptr, a.ws + a.ws_bytes,
-                              up256(select_ws_bytes(g)), stream);
-        if (rc != STC_OK) return rc;
-        ids = reinterpret_cast<const int32_t*>(a.ids);
+        rc = stc_decode_step(shape, cache, a.q, token_budget, a.max_pages, reinterpret_cast<int32_t*>(a.ids),
+                             reinterpret_cast<int32_t*>(a.npages), sm_scale, reinterpret_cast<float*>(a.out), nullptr,
+                             a.ws + a.ws_bytes, up256(select_ws_bytes(g)), a.ws, a.ws_bytes, stream);
+    } else {
+        rc = stc_decode_attn(shape, cache, a.q, nullptr, nullptr, a.max_pages, sm_scale,
+                             reinterpret_cast<float*>(a.out), nullptr, a.ws, a.ws_bytes, stream);
     }
-    rc = stc_decode_attn(shape, cache, a.q, ids, reinterpret_cast<const int32_t*>(a.npages), a.max_pages,
-                         sm_scale, reinterpret_cast<float*>(a.out), nullptr, a.ws, a.ws_bytes, stream);
     if (rc != STC_OK) return rc;
     cudaError_t e = cudaMemcpyAsync(out_host, a.out, (size_t)g.B * g.Hq * kHeadDim * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(status_host, a.ws, 4, cudaMemcpyDeviceToHost, st);
