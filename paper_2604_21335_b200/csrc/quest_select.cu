@@ -76,7 +76,8 @@ constexpr size_t kRingBytes = (size_t)kDepth * kThreads * 32;
 //   3. ordered compaction: keys above the threshold, plus the first
 //      k - #above keys equal to it in index order, ballot-ranked per warp.
 constexpr int kRankMax = 64;
-constexpr int kTopkSmemWords = 256 /*hist*/ + kRankMax /*candidates*/ + 2 * kWarps + 8 /*scalars*/;
+constexpr int kMaxWarps = 16;                 // the selection code runs with 256 or 512 threads
+constexpr int kTopkSmemWords = 256 /*hist*/ + kRankMax /*candidates*/ + 2 * kMaxWarps + 8 /*scalars*/;
 constexpr int kSmemKeys = (int)(kRingBytes / 4);
 
 // Bound of one page in the declared fp32 order, by one half-warp (lane l of the half owns
@@ -107,20 +108,22 @@ constexpr int kAmbMax = 2048;
 // scored exactly, ranked by (exact score descending, index ascending), and the best of them
 // fill the remaining places.  Returns false (nothing written) when more than kAmbMax pages
 // fall in between; u may be overwritten.
+template <int NT>
 __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int32_t* __restrict__ ids,
                                         uint32_t* __restrict__ skeys, uint32_t* __restrict__ sh,
                                         const FilterCtx* __restrict__ f) {
+    constexpr int NW = NT / 32;
     __syncthreads();                              // nobody still reads what an earlier selection left in the scratch
     uint32_t* hist = sh;
     uint32_t* cbuf = sh + 256;
-    uint32_t* sc = sh + 256 + kRankMax;         // [kWarps] warp mins, [kWarps] warp maxs / totals, then results
+    uint32_t* sc = sh + 256 + kRankMax;         // [NW] warp mins, [NW] warp maxs / totals, then results
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // Warp w owns the index block [w*per_warp, (w+1)*per_warp); a lane visits groups of four
     // consecutive keys (one 16-byte read), group j*32 + lane in pass j.  Slots past n hold key 0,
     // which is below every real key, so it can never be selected (k < n).
-    const int per_warp = ((n + kWarps * 128 - 1) / (kWarps * 128)) * 128;
+    const int per_warp = ((n + NW * 128 - 1) / (NW * 128)) * 128;
     const int J = per_warp / 128;                // groups per lane
-    const int padded = per_warp * kWarps;
+    const int padded = per_warp * NW;
     const unsigned lt = (1u << lane) - 1u;
     const bool staged = padded <= kSmemKeys;
 
@@ -130,11 +133,11 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
         // up to eight groups per thread in flight (one round trip to L2 for 8192 keys)
         const bool vec = (reinterpret_cast<uintptr_t>(u) & 15u) == 0;
 #pragma unroll 1
-        for (int g0 = tid; g0 < padded / 4; g0 += 8 * kThreads) {
+        for (int g0 = tid; g0 < padded / 4; g0 += 8 * NT) {
             uint4 raw[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int i = 4 * (g0 + e * kThreads);
+                const int i = 4 * (g0 + e * NT);
                 raw[e] = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);   // -NaN: key 0
                 if (vec && i + 3 < n) {
                     raw[e] = __ldcg(reinterpret_cast<const uint4*>(u + i));
@@ -147,7 +150,7 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
             }
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int i = 4 * (g0 + e * kThreads);
+                const int i = 4 * (g0 + e * NT);
                 if (i >= padded) continue;
                 const uint32_t w4[4] = {raw[e].x, raw[e].y, raw[e].z, raw[e].w};
                 uint32_t x[4];
@@ -183,10 +186,10 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
         });
     kmn = __reduce_min_sync(0xFFFFFFFFu, kmn);
     kmx = __reduce_max_sync(0xFFFFFFFFu, kmx);
-    if (lane == 0) { sc[warp] = kmn; sc[kWarps + warp] = kmx; }
+    if (lane == 0) { sc[warp] = kmn; sc[NW + warp] = kmx; }
     __syncthreads();
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) { kmn = min(kmn, sc[w2]); kmx = max(kmx, sc[kWarps + w2]); }
+    for (int w2 = 0; w2 < NW; ++w2) { kmn = min(kmn, sc[w2]); kmx = max(kmx, sc[NW + w2]); }
 
     // ---- 2. k-th largest key -----------------------------------------------------------------
     int bits_left = 32 - __clz(kmn ^ kmx);       // low bits that differ somewhere (0: all keys equal)
@@ -200,12 +203,12 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
         __syncthreads();                          // previous readers of hist / scalars are done
         if (cand <= (uint32_t)kRankMax) {
             // gather the candidates and rank them directly
-            if (tid == 0) sc[2 * kWarps] = 0u;
+            if (tid == 0) sc[2 * NW] = 0u;
             __syncthreads();
             for_each([&](const uint32_t (&x)[4], int) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (x[e] != 0u && (x[e] & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[2 * kWarps], 1u)] = x[e];
+                    if (x[e] != 0u && (x[e] & fixed_mask) == fixed_val) cbuf[atomicAdd(&sc[2 * NW], 1u)] = x[e];
             });
             __syncthreads();
             if ((uint32_t)tid < cand) {
@@ -213,10 +216,10 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
                 uint32_t g = 0, e = 0;
 #pragma unroll 4
                 for (uint32_t i = 0; i < cand; ++i) { const uint32_t y = cbuf[i]; g += y > x; e += y == x; }
-                if (g < krem && krem <= g + e) sc[2 * kWarps + 1] = x;   // every thread that qualifies holds the same key
+                if (g < krem && krem <= g + e) sc[2 * NW + 1] = x;   // every thread that qualifies holds the same key
             }
             __syncthreads();
-            tau = sc[2 * kWarps + 1];
+            tau = sc[2 * NW + 1];
             break;
         }
         const int nb = bits_left < 8 ? bits_left : 8, shift = bits_left - nb;
@@ -239,15 +242,15 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     if (run < krem && krem <= run + c8[i]) {
-                        sc[2 * kWarps + 2] = 255 - 8 * lane - i; sc[2 * kWarps + 3] = krem - run; sc[2 * kWarps + 4] = c8[i];
+                        sc[2 * NW + 2] = 255 - 8 * lane - i; sc[2 * NW + 3] = krem - run; sc[2 * NW + 4] = c8[i];
                     }
                     run += c8[i];
                 }
             }
         }
         __syncthreads();
-        const uint32_t digit = sc[2 * kWarps + 2];
-        krem = sc[2 * kWarps + 3]; cand = sc[2 * kWarps + 4];
+        const uint32_t digit = sc[2 * NW + 2];
+        krem = sc[2 * NW + 3]; cand = sc[2 * NW + 4];
         fixed_mask |= dmask << shift;
         fixed_val |= digit << shift;
         bits_left = shift;
@@ -259,7 +262,7 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
         const float tf = key_float(tau), pad = 2.0f * f->delta;
         const uint32_t key_hi = float_key(tf + pad), key_lo = float_key(tf - pad);
         __syncthreads();
-        if (tid == 0) { sc[2 * kWarps] = 0u; sc[2 * kWarps + 1] = 0u; }
+        if (tid == 0) { sc[2 * NW] = 0u; sc[2 * NW + 1] = 0u; }
         __syncthreads();
         uint32_t n_in = 0;
         for_each([&](const uint32_t (&x)[4], int i0) {
@@ -267,22 +270,22 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
             for (int e = 0; e < 4; ++e) {
                 if (x[e] > key_hi) ++n_in;
                 else if (x[e] >= key_lo && x[e] != 0u) {
-                    const uint32_t pos = atomicAdd(&sc[2 * kWarps], 1u);
+                    const uint32_t pos = atomicAdd(&sc[2 * NW], 1u);
                     if (pos < (uint32_t)kAmbMax) f->amb_idx[pos] = i0 + e;
                 }
             }
         });
         n_in = __reduce_add_sync(0xFFFFFFFFu, n_in);
-        if (lane == 0) atomicAdd(&sc[2 * kWarps + 1], n_in);
+        if (lane == 0) atomicAdd(&sc[2 * NW + 1], n_in);
         __syncthreads();
-        const int n_amb = (int)sc[2 * kWarps];
-        const int need = k - (int)sc[2 * kWarps + 1];      // 1 <= need <= n_amb
+        const int n_amb = (int)sc[2 * NW];
+        const int need = k - (int)sc[2 * NW + 1];      // 1 <= need <= n_amb
         if (n_amb > kAmbMax) return false;
         {
             const int half = lane >> 4, l = lane & 15;
             const unsigned hm = 0xFFFFu << (16 * half);
 #pragma unroll 1
-            for (int e0 = 0; e0 < n_amb; e0 += 2 * kWarps) {
+            for (int e0 = 0; e0 < n_amb; e0 += 2 * NW) {
                 const int e = e0 + warp * 2 + half;
                 const int idx = f->amb_idx[min(e, n_amb - 1)];
                 const float sx = exact_page_score(f->kmin + (size_t)idx * kOctets, f->kmax + (size_t)idx * kOctets,
@@ -292,7 +295,7 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
         }
         __syncthreads();
 #pragma unroll 1
-        for (int e = tid; e < n_amb; e += kThreads) {
+        for (int e = tid; e < n_amb; e += NT) {
             const uint32_t kx = f->amb_key[e];
             const int ix = f->amb_idx[e];
             int rank = 0;
@@ -320,12 +323,12 @@ __device__ __noinline__ bool block_topk(float* __restrict__ u, int n, int k, int
     gt = __reduce_add_sync(0xFFFFFFFFu, gt);
     eq = __reduce_add_sync(0xFFFFFFFFu, eq);
     __syncthreads();
-    if (lane == 0) { sc[warp] = gt; sc[kWarps + warp] = eq; }
+    if (lane == 0) { sc[warp] = gt; sc[NW + warp] = eq; }
     __syncthreads();
     uint32_t run_gt = 0, run_eq = 0, all_gt = 0;
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) {
-        if (w2 < warp) { run_gt += sc[w2]; run_eq += sc[kWarps + w2]; }
+    for (int w2 = 0; w2 < NW; ++w2) {
+        if (w2 < warp) { run_gt += sc[w2]; run_eq += sc[NW + w2]; }
         all_gt += sc[w2];
     }
     const uint32_t ties = (uint32_t)k - all_gt;   // keys equal to tau still to take, lowest indices first
@@ -430,11 +433,11 @@ __device__ __noinline__ float exact_page_score(const uint4* __restrict__ kmin_ro
 }
 
 // ---- the tensor-core scan ------------------------------------------------------------------
-// A warp owns a tile of 16 consecutive pages; a unit is the 8 tiles of a CTA (128 pages).
+// A warp owns a tile of 16 consecutive pages; a unit is the 16 tiles of a CTA (256 pages).
 // A tile is two contiguous 4 KiB blocks (16 rows of kmax, 16 rows of kmin): lane 0 brings them
-// into one of the warp's kFDepth ring slots with two bulk asynchronous copies that signal the
-// slot's mbarrier, two tiles ahead of the one being reduced, and the copies run on across the
-// boundaries between problems; nothing waits on another warp.  Every wait on an mbarrier is
+// into the warp's ring slot with two bulk asynchronous copies that signal the slot's mbarrier
+// (sixteen warps per SM, so sixteen tiles are in flight or being reduced at any time), and the
+// copies run on across the boundaries between problems; nothing waits on another warp.  Every wait on an mbarrier is
 // bounded: a wait that expires records STC_ERR_TIMEOUT in the workspace status word and the
 // warp stops issuing copies and skips its arithmetic (the page lists of the call are then
 // unspecified, still valid ids).
@@ -450,12 +453,14 @@ __device__ __noinline__ float exact_page_score(const uint4* __restrict__ kmin_ro
 constexpr int kFilterMinGq = 2;               // single-head problems stay on the fp32 pipes
 constexpr int kFilterMinPages = 4096;         // pages per problem from which the filtered scan is the faster one
 constexpr int kFilterMinPagesSplit = 1024;    // ... with more than four query heads per KV head
-constexpr int kFDepth = 2;                                       // tiles in flight per warp
+constexpr int kFThreads = 512;                                   // one CTA per SM, 16 warps
+constexpr int kFWarps = kFThreads / 32;
+constexpr int kFDepth = 1;                                       // ring slots per warp (16 tiles in flight per SM)
 constexpr int kFCtasPerSm = 1;
 constexpr uint32_t kFTileBytes = 16u * 512u;                     // 8 KiB per tile: kmax rows | kmin rows
-constexpr size_t kFRingBytes = (size_t)kWarps * kFDepth * kFTileBytes;   // 128 KiB
+constexpr size_t kFRingBytes = (size_t)kFWarps * kFDepth * kFTileBytes;  // 128 KiB
 constexpr unsigned long long kFWaitLimitNs = 1000000000ull;
-constexpr int kFUnitPages = kWarps * 16;
+constexpr int kFUnitPages = kFWarps * 16;
 constexpr float kMarginRel = 1.0f / 8192.0f;   // 2^-13 of sum|term|: far above the 2^-24-per-add error of either sum
 
 // Shared memory of the selection behind the copy ring (the ring keeps streaming the next
@@ -485,6 +490,7 @@ static_assert(kFSmemBytes <= 227 * 1024 - 2048, "ring + selection scratch fit on
 //      (exact score descending, page ascending); the verdicts are written into the staged keys;
 //   D. one pass writes the selected pages in ascending order (ballot ranks inside a warp's
 //      contiguous block, block offsets from the per-warp counts).
+template <int NT>
 __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int n, int k, int32_t* __restrict__ ids,
                                                 uint32_t* __restrict__ sm, uint32_t* __restrict__ sc,
                                                 uint32_t key_min, uint32_t key_max,
@@ -494,21 +500,22 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
     int32_t* cidx = reinterpret_cast<int32_t*>(sm + kSelCidx);
     uint32_t* ckey = sm + kSelCkey;
     uint32_t* amb = sm + kSelAmb;
-    // scalars: sc[0..7] warp totals of the bin scan, sc[8..15] selected pages per warp block, then
-    enum { kCnt = 16, kTau, kBin, kAbove, kNin, kNamb };
+    constexpr int NW = NT / 32, BPT = kHistBins / NT;      // warps; histogram bins per thread in the bin scan
+    // scalars: sc[0..NW) warp totals of the bin scan, sc[NW..2NW) selected pages per warp block, then
+    enum { kCnt = 2 * NW, kTau, kBin, kAbove, kNin, kNamb };
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bits_left = 32 - __clz(key_min ^ key_max);
     if (bits_left == 0 || n > kSmemKeys) return false;
     const int nb = bits_left < kHistBits ? bits_left : kHistBits, shift = bits_left - nb;
     const uint32_t dmask = (1u << nb) - 1u;
     const uint32_t fixed = bits_left >= 32 ? 0u : (key_max & ~((1u << bits_left) - 1u));
-    const int per_warp = ((n + kWarps * 128 - 1) / (kWarps * 128)) * 128;
+    const int per_warp = ((n + NW * 128 - 1) / (NW * 128)) * 128;
     const int J = per_warp / 128;
     const unsigned lt = (1u << lane) - 1u;
     const bool vec = (reinterpret_cast<uintptr_t>(u) & 15u) == 0;
 
-    for (int i = tid; i < kHistBins; i += kThreads) hist[i] = 0u;
-    if (tid < 32) sc[tid] = 0u;
+    for (int i = tid; i < kHistBins; i += NT) hist[i] = 0u;
+    if (tid < 2 * NW + 8) sc[tid] = 0u;
     __syncthreads();
 
     // ---- A. stage + histogram --------------------------------------------------------------------
@@ -545,23 +552,23 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
     }
     __syncthreads();
 
-    // ---- bin of the k-th largest key: thread t owns bins 2047 - 8t - i, i = 0..7 (descending) ----
+    // ---- bin of the k-th largest key: thread t owns bins 2047 - BPT t - i, i = 0..BPT-1 (descending) ----
     {
-        uint32_t c8[8], sum = 0;
+        uint32_t c8[BPT], sum = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { c8[i] = hist[kHistBins - 1 - 8 * tid - i]; sum += c8[i]; }
+        for (int i = 0; i < BPT; ++i) { c8[i] = hist[kHistBins - 1 - BPT * tid - i]; sum += c8[i]; }
         const uint32_t incl_w = warp_incl_scan(sum, lane);
         if (lane == 31) sc[warp] = incl_w;
         __syncthreads();
         uint32_t before = 0;
 #pragma unroll
-        for (int w2 = 0; w2 < kWarps; ++w2) if (w2 < warp) before += sc[w2];
+        for (int w2 = 0; w2 < NW; ++w2) if (w2 < warp) before += sc[w2];
         const uint32_t incl = before + incl_w, excl = incl - sum;
         if (excl < (uint32_t)k && (uint32_t)k <= incl) {
             uint32_t run = excl;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (run < (uint32_t)k && (uint32_t)k <= run + c8[i]) { sc[kBin] = kHistBins - 1 - 8 * tid - i; sc[kAbove] = run; }
+            for (int i = 0; i < BPT; ++i) {
+                if (run < (uint32_t)k && (uint32_t)k <= run + c8[i]) { sc[kBin] = kHistBins - 1 - BPT * tid - i; sc[kAbove] = run; }
                 run += c8[i];
             }
         }
@@ -594,14 +601,14 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
             }
         }
         wc = __reduce_add_sync(0xFFFFFFFFu, wc);
-        if (lane == 0) sc[8 + warp] = wc;
+        if (lane == 0) sc[NW + warp] = wc;
     }
     __syncthreads();
     const int ncand = (int)sc[kCnt];
     if (ncand > kCandMax) return false;                                  // (cannot happen: the bins were counted)
 
     // ---- C. the k-th largest approximate key, then the verdict on every candidate -----------------
-    for (int e = tid; e < ncand; e += kThreads) {
+    for (int e = tid; e < ncand; e += NT) {
         const uint32_t x = ckey[e];
         if ((int)((x >> shift) & dmask) != bin) continue;
         uint32_t gt = 0, eq = 0;
@@ -618,12 +625,12 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
     const uint32_t lo_edge = bin >= 1 ? (fixed | ((uint32_t)(bin - 1) << shift)) : 0u;
     const uint32_t hi_edge = (uint32_t)(bin + 2) <= dmask ? (fixed | (((uint32_t)(bin + 2) << shift) - 1u)) : 0xFFFFFFFEu;
     if ((bin >= 2 && key_lo < lo_edge) || ((uint32_t)(bin + 2) <= dmask && key_hi > hi_edge)) return false;
-    for (int e = tid; e < ncand; e += kThreads) {
+    for (int e = tid; e < ncand; e += NT) {
         const uint32_t x = ckey[e];
         const int ix = cidx[e];
         if (x > key_hi) {                                                // certainly selected
             skeys[ix] = 0xFFFFFFFFu;
-            atomicAdd(&sc[8 + ix / per_warp], 1u);
+            atomicAdd(&sc[NW + ix / per_warp], 1u);
             atomicAdd(&sc[kNin], 1u);
         } else if (x >= key_lo) {
             amb[atomicAdd(&sc[kNamb], 1u)] = (uint32_t)e;                // settled below
@@ -639,7 +646,7 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
         const int half = lane >> 4, l = lane & 15;
         const unsigned hm = 0xFFFFu << (16 * half);
 #pragma unroll 1
-        for (int e0 = 0; e0 < n_amb; e0 += 2 * kWarps) {
+        for (int e0 = 0; e0 < n_amb; e0 += 2 * NW) {
             const int e = e0 + warp * 2 + half;
             const int ce = (int)amb[min(e, n_amb - 1)];
             const int idx = cidx[ce];
@@ -649,7 +656,7 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
         }
     }
     __syncthreads();
-    for (int e = tid; e < n_amb; e += kThreads) {
+    for (int e = tid; e < n_amb; e += NT) {
         const uint32_t kx = ckey[amb[e]];
         const int ix = cidx[amb[e]];
         int rank = 0;
@@ -660,14 +667,14 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
         }
         const bool chosen = rank < need;
         skeys[ix] = chosen ? 0xFFFFFFFFu : 0u;
-        if (chosen) atomicAdd(&sc[8 + ix / per_warp], 1u);
+        if (chosen) atomicAdd(&sc[NW + ix / per_warp], 1u);
     }
     __syncthreads();
 
     // ---- D. ordered write ---------------------------------------------------------------------------
     uint32_t base = 0, all = 0;
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) { if (w2 < warp) base += sc[8 + w2]; all += sc[8 + w2]; }
+    for (int w2 = 0; w2 < NW; ++w2) { if (w2 < warp) base += sc[NW + w2]; all += sc[NW + w2]; }
     if (all != (uint32_t)k) return false;                                // (cannot happen; u is still intact)
 #pragma unroll 2
     for (int j = 0; j < J; ++j) {
@@ -709,7 +716,7 @@ struct ProblemStats {
 };
 
 template <int GQ>
-__global__ void __launch_bounds__(kThreads, kFCtasPerSm)
+__global__ void __launch_bounds__(kFThreads, kFCtasPerSm)
 quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ kmax,
                     const uint4* __restrict__ q, const int32_t* __restrict__ seq_len, int Hq, int Hkv,
                     int T, int P, int token_budget, int n_recent, int max_pages, int32_t* __restrict__ page_ids,
@@ -717,7 +724,7 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                     int32_t* __restrict__ status, int units_per_problem, long long total_units) {
     extern __shared__ __align__(128) uint32_t ring_mem[];
     __shared__ uint32_t s_topk[kTopkSmemWords];
-    __shared__ __align__(8) unsigned long long s_bars[kWarps * kFDepth];
+    __shared__ __align__(8) unsigned long long s_bars[kFWarps * kFDepth];
     __shared__ int s_last;
     uint32_t* sel_mem = ring_mem + kFRingBytes / 4;
 
@@ -770,7 +777,7 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             if (nv > 0 && !dead && lane == 0) {
                 const size_t row = (size_t)si.problem * P + page0;
                 const uint32_t dst = ring + (uint32_t)slot_issue * kFTileBytes, bar = bars + 8u * slot_issue;
-                if (reuse) fence_proxy_async();   // the slot's earlier reads precede the new writes
+                (void)reuse;   // the slot's earlier reads have returned their data (the warp has used it)
                 mbar_expect_tx(bar, (uint32_t)nv * 512u);
                 bulk_g2s(dst, kmax + row * kOctets, (uint32_t)nv * 256u, bar);
                 bulk_g2s(dst + 4096u, kmin + row * kOctets, (uint32_t)nv * 256u, bar);
@@ -793,7 +800,7 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
         if (sg.trivial) {                          // no scores needed
             if (sg.u_begin == 0) {
                 int32_t* ids = page_ids + (size_t)problem * max_pages;
-                for (int i = tid; i < k_pg; i += kThreads) ids[i] = i;
+                for (int i = tid; i < k_pg; i += kFThreads) ids[i] = i;
                 if (tid == 0) n_pages[problem] = max(k_pg, 0);
             }
             continue;
@@ -802,8 +809,8 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
         const size_t row0 = (size_t)problem * P;
         const uint4* q_heads = q + ((size_t)b * Hq + (size_t)hk * GQ) * kOctets;
 
-        // ---- query fragments of column n = g: chunks t + 4j of q+ and q- (and |q-|) ----
-        uint32_t qp[4][4], qn[4][4], qa[4][4];
+        // ---- query fragments of column n = g: chunks t + 4j of q+ and q- ----
+        uint32_t qp[4][4], qn[4][4];
         {
             const uint4* qrow = q_heads + (size_t)(g < GQ ? g : g % GQ) * kOctets;
 #pragma unroll
@@ -815,7 +822,6 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                     const uint32_t neg = ((w[c] >> 15) & 0x00010001u) * 0xFFFFu;   // 0xFFFF in the negative halves
                     qn[j][c] = w[c] & neg;
                     qp[j][c] = w[c] & ~neg;
-                    qa[j][c] = qn[j][c] & kAbs;
                 }
             }
         }
@@ -846,11 +852,11 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                     mma_bf16_16816(sx, x0.x, x8.x, x0.y, x8.y, qp[j][0], qp[j][1]);
                     mma_bf16_16816(sn, n0.x, n8.x, n0.y, n8.y, qn[j][0], qn[j][1]);
                     mma_bf16_16816(ax, x0.x & kAbs, x8.x & kAbs, x0.y & kAbs, x8.y & kAbs, qp[j][0], qp[j][1]);
-                    mma_bf16_16816(an, n0.x & kAbs, n8.x & kAbs, n0.y & kAbs, n8.y & kAbs, qa[j][0], qa[j][1]);
+                    mma_bf16_16816(an, n0.x & kAbs, n8.x & kAbs, n0.y & kAbs, n8.y & kAbs, qn[j][0] & kAbs, qn[j][1] & kAbs);
                     mma_bf16_16816(sx, x0.z, x8.z, x0.w, x8.w, qp[j][2], qp[j][3]);
                     mma_bf16_16816(sn, n0.z, n8.z, n0.w, n8.w, qn[j][2], qn[j][3]);
                     mma_bf16_16816(ax, x0.z & kAbs, x8.z & kAbs, x0.w & kAbs, x8.w & kAbs, qp[j][2], qp[j][3]);
-                    mma_bf16_16816(an, n0.z & kAbs, n8.z & kAbs, n0.w & kAbs, n8.w & kAbs, qa[j][2], qa[j][3]);
+                    mma_bf16_16816(an, n0.z & kAbs, n8.z & kAbs, n0.w & kAbs, n8.w & kAbs, qn[j][2] & kAbs, qn[j][3] & kAbs);
                 }
                 __syncwarp();                            // every lane has read the slot
                 issue(true);                             // refills the slot just consumed
@@ -913,13 +919,13 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                 f.amb_key = sel_mem + kSmemKeys + kAmbMax;
                 float* u = scores + row0;
                 const uint32_t key_max = __ldcg(st.keymax + problem), key_min = ~__ldcg(st.keymin_inv + problem);
-                if (!filter_select_fast(u, np - w, k_pg - w, ids, sel_mem, s_topk, key_min, key_max, &f) &&
-                    !block_topk(u, np - w, k_pg - w, ids, sel_mem, s_topk, &f)) {
+                if (!filter_select_fast<kFThreads>(u, np - w, k_pg - w, ids, sel_mem, s_topk, key_min, key_max, &f) &&
+                    !block_topk<kFThreads>(u, np - w, k_pg - w, ids, sel_mem, s_topk, &f)) {
                     // too many pages within the margin (many equal pages): score every page exactly instead
                     const int half = lane >> 4, l = lane & 15;
                     const unsigned hm = 0xFFFFu << (16 * half);
 #pragma unroll 1
-                    for (int p0 = 0; p0 < np - w; p0 += 2 * kWarps) {
+                    for (int p0 = 0; p0 < np - w; p0 += 2 * kFWarps) {
                         const int p = p0 + warp * 2 + half;
                         const int pc = min(p, np - w - 1);
                         const float sxp = exact_page_score(f.kmin + (size_t)pc * kOctets, f.kmax + (size_t)pc * kOctets,
@@ -928,10 +934,10 @@ quest_filter_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
                     }
                     __threadfence_block();
                     __syncthreads();
-                    block_topk(u, np - w, k_pg - w, ids, sel_mem, s_topk, nullptr);
+                    block_topk<kFThreads>(u, np - w, k_pg - w, ids, sel_mem, s_topk, nullptr);
                 }
             }
-            for (int i = tid; i < w; i += kThreads) ids[k_pg - w + i] = np - w + i;
+            for (int i = tid; i < w; i += kFThreads) ids[k_pg - w + i] = np - w + i;
             if (tid == 0) n_pages[problem] = k_pg;
         }
     }
@@ -1077,7 +1083,7 @@ quest_select_kernel(const uint4* __restrict__ kmin, const uint4* __restrict__ km
             // the copy ring is idle here (all copies have landed): it stages the keys
             // the local window: the last w pages are kept, the rest of the budget goes to the pages before them
             const int w = min(max(n_recent, 0), k_pg);
-            if (k_pg > w) block_topk(scores + row0, np - w, k_pg - w, ids, ring_mem, s_topk, nullptr);
+            if (k_pg > w) block_topk<kThreads>(scores + row0, np - w, k_pg - w, ids, ring_mem, s_topk, nullptr);
             for (int i = tid; i < w; i += kThreads) ids[k_pg - w + i] = np - w + i;
             if (tid == 0) n_pages[problem] = k_pg;
         }
@@ -1130,7 +1136,7 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
         if (filter) {                                                                                \
             cudaFuncSetAttribute(quest_filter_kernel<GQ_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                  (int)kFSmemBytes);                                                  \
-            quest_filter_kernel<GQ_><<<(unsigned)grid, kThreads, kFSmemBytes, st>>>(                 \
+            quest_filter_kernel<GQ_><<<(unsigned)grid, kFThreads, kFSmemBytes, st>>>(                \
                 static_cast<const uint4*>(kmin), static_cast<const uint4*>(kmax),                    \
                 static_cast<const uint4*>(q), g.seq_len, g.Hq, g.Hkv, g.T, g.P, token_budget,        \
                 n_recent_pages, max_pages, page_ids, n_pages, scores, stats, status,                 \
