@@ -483,8 +483,8 @@ static_assert(kFSmemBytes <= 227 * 1024 - 2048, "ring + selection scratch fit on
 // does not handle turns up, and the caller then takes block_topk.
 //   A. one pass stages the keys and builds the histogram of the top kHistBits bits on which the
 //      problem's keys differ; a block-wide scan of the bins finds the bin b of the k-th largest key;
-//   B. one pass gathers the keys of bins b-1, b, b+1 (the k-th key and everything within the
-//      margin of it -- checked, else false) and counts, per warp, the keys in the bins above;
+//   B. one pass gathers the keys of the bins around b that can hold a key within the margin of the
+//      k-th key, and counts, per warp, the keys in the bins above them;
 //   C. the k-th largest key t is ranked among the candidates; candidates above t + 2 delta are
 //      selected, those below t - 2 delta are not, the rest are scored exactly and ranked by
 //      (exact score descending, page ascending); the verdicts are written into the staged keys;
@@ -576,9 +576,19 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
     }
     const int bin = (int)sc[kBin];
     const uint32_t above = sc[kAbove];                                   // keys in the bins above `bin`
-    const uint32_t cnt_b = hist[bin];
-    const uint32_t cnt_up = bin + 1 < kHistBins ? hist[bin + 1] : 0u, cnt_dn = bin >= 1 ? hist[bin - 1] : 0u;
-    if (cnt_b + cnt_up + cnt_dn > (uint32_t)kCandMax) return false;
+    // The k-th key t lies in `bin`, so every key within 2 delta of it lies between (lowest value of the bin)
+    // - 2 delta and (highest value of the bin) + 2 delta: the bins d_lo..d_hi of those two keys (keys outside
+    // the problem's own range do not exist) hold the k-th key and the whole window around it.
+    const float pad = 2.0f * f->delta;
+    const uint32_t bin_lo_key = fixed | ((uint32_t)bin << shift);
+    const uint32_t bin_hi_key = bin_lo_key | ((1u << shift) - 1u);
+    const uint32_t k_lo = max(float_key(key_float(bin_lo_key) - pad), key_min);
+    const uint32_t k_hi = min(float_key(key_float(bin_hi_key) + pad), key_max);
+    const int d_lo = (int)((k_lo >> shift) & dmask), d_hi = (int)((k_hi >> shift) & dmask);
+    if (d_lo > bin || d_hi < bin || d_hi - d_lo > 64) return false;      // (non-finite scores)
+    uint32_t cnt_gathered = 0, cnt_up = 0;                               // keys in d_lo..d_hi; of them, above `bin`
+    for (int d = d_lo; d <= d_hi; ++d) { const uint32_t c = hist[d]; cnt_gathered += c; if (d > bin) cnt_up += c; }
+    if (cnt_gathered > (uint32_t)kCandMax) return false;
     const uint32_t krem = (uint32_t)k - above;                           // rank of the k-th key inside its bin
 
     // ---- B. gather the candidates, count the certainly selected keys per warp block ---------------
@@ -593,8 +603,8 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
             for (int e = 0; e < 4; ++e) {
                 if (x[e] == 0u) continue;
                 const int d = (int)((x[e] >> shift) & dmask);
-                if (d > bin + 1) ++wc;
-                else if (d >= bin - 1) {
+                if (d > d_hi) ++wc;
+                else if (d >= d_lo) {
                     const uint32_t pos = atomicAdd(&sc[kCnt], 1u);
                     if (pos < (uint32_t)kCandMax) { cidx[pos] = i0 + e; ckey[pos] = x[e]; }
                 }
@@ -606,6 +616,11 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
     __syncthreads();
     const int ncand = (int)sc[kCnt];
     if (ncand > kCandMax) return false;                                  // (cannot happen: the bins were counted)
+    // the metadata rows of the candidates are wanted in a moment by the exact re-scoring: start them towards L2
+    for (int e = tid; e < 4 * ncand; e += NT) {
+        const char* row = reinterpret_cast<const char*>(((e & 2) ? f->kmax : f->kmin) + (size_t)cidx[e >> 2] * kOctets);
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(row + 128 * (e & 1)));
+    }
 
     // ---- C. the k-th largest approximate key, then the verdict on every candidate -----------------
     for (int e = tid; e < ncand; e += NT) {
@@ -614,17 +629,15 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
         uint32_t gt = 0, eq = 0;
 #pragma unroll 4
         for (int o = 0; o < ncand; ++o) { const uint32_t y = ckey[o]; gt += y > x; eq += y == x; }
-        gt -= cnt_up;                                                    // the keys of bin + 1 are all larger
+        gt -= cnt_up;                                                    // the gathered keys of the bins above are all larger
         if (gt < krem && krem <= gt + eq) sc[kTau] = x;                  // every thread that qualifies holds the same key
     }
     __syncthreads();
     const uint32_t tau = sc[kTau];
-    const float tf = key_float(tau), pad = 2.0f * f->delta;
+    const float tf = key_float(tau);
     const uint32_t key_hi = float_key(tf + pad), key_lo = float_key(tf - pad);
-    // the gathered bins must hold every key within the margin of tau
-    const uint32_t lo_edge = bin >= 1 ? (fixed | ((uint32_t)(bin - 1) << shift)) : 0u;
-    const uint32_t hi_edge = (uint32_t)(bin + 2) <= dmask ? (fixed | (((uint32_t)(bin + 2) << shift) - 1u)) : 0xFFFFFFFEu;
-    if ((bin >= 2 && key_lo < lo_edge) || ((uint32_t)(bin + 2) <= dmask && key_hi > hi_edge)) return false;
+    // keys above hi_edge (the largest key of bin d_hi) were counted as certainly selected
+    const uint32_t hi_edge = min(fixed | ((uint32_t)d_hi << shift) | ((1u << shift) - 1u), 0xFFFFFFFEu);
     for (int e = tid; e < ncand; e += NT) {
         const uint32_t x = ckey[e];
         const int ix = cidx[e];
