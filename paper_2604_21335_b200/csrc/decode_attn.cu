@@ -172,15 +172,11 @@ decode_attn_kernel(const AttnArgs a) {
         }
     };
 
-    // ---- the pages in flight: one set of registers per stage, written when the stage is issued and
-    //      read when it is consumed kStages pages later (nothing is shifted in between, so the loads
-    //      of the mask and the offset have a whole turn of the ring to arrive) -------------------------
+    // ---- the pages in flight: a register FIFO, oldest first (uniform across the warp except mask) ----
     struct InFlight {
         int nv;              // valid tokens; 0 = nothing to attend at this position
         uint32_t chunks;     // 16-byte chunks of the value span present in the stage
         uint32_t mask;       // lanes 0..15: group mask of token `lane`
-        uint32_t pre;        // lanes 0..15: groups stored before token `lane` (absolute offset)
-        uint32_t first;      // first packed group of the page (clipped to the store)
     };
     uint32_t phase = 0;                          // bit s = parity to wait for on stage s
 
@@ -190,53 +186,34 @@ decode_attn_kernel(const AttnArgs a) {
     int p_issue = (int)(x_lo / mp);              // its problem
     int slot_issue = (int)(x_lo - (long long)p_issue * mp);
 
-    InFlight f[kStages];                         // f[s] = the page in stage s
-#pragma unroll
-    for (int i = 0; i < kStages; ++i) f[i] = InFlight{0, 0u, 0u, 0u, 0u};
-    // Bring position x_issue into stage s.  The loads of the page's token masks and offsets go
-    // straight into stage s's own registers (one predicated load per stage, only stage s's is live),
-    // so that no instruction touches their result before the page is consumed.
-    auto issue = [&](int s) {
-        int nv = 0;
-        uint32_t chunks = 0u;
-        if (x_issue < x_hi) {
-            if (x_issue - win_base >= 32) { win_base = x_issue; fill_window(win_base); }
-            const int src = (int)(x_issue - win_base);
-            const int page = __shfl_sync(0xFFFFFFFFu, win.page, src);
-            const int nvp = __shfl_sync(0xFFFFFFFFu, win.n_valid, src);
-            const uint32_t first = __shfl_sync(0xFFFFFFFFu, win.first, src);
-            const uint32_t groups = __shfl_sync(0xFFFFFFFFu, win.groups, src);
-            if (page >= 0) {
-                const size_t row0 = (size_t)p_issue * a.T + (size_t)page * kPage;
-                const uint16_t* mp_ = a.v_mask + row0 + lane;
-                const uint32_t* op_ = a.v_offs + (size_t)p_issue * (a.T + 1) + (size_t)page * kPage + lane;
-#pragma unroll
-                for (int i = 0; i < kStages; ++i)
-                    if (i == s && lane < nvp) {
-                        f[i].mask = *mp_;
-                        f[i].pre = *op_;             // absolute; made relative to the page when it is consumed
-                    }
-                nv = nvp;
-                chunks = groups * OPG;
-                if (lane == 0) {
-                    const uint32_t kb = (uint32_t)nvp * kRowBytes, vb = groups * kGroupBytes;
-                    const uint32_t bar = bars + 8 * s, dst = ring + (uint32_t)s * kStageBytes;
-                    // (the stage's earlier reads have returned their data -- the warp computed with it --
-                    // so the new copies may overwrite it)
-                    mbar_expect_tx(bar, kb + vb);
-                    bulk_g2s(dst, a.k + row0 * kRowBytes, kb, bar);
-                    if (vb)
-                        bulk_g2s(dst + kKeyBytes,
-                                 a.v_packed + ((size_t)p_issue * a.cap_groups + first) * kGroupBytes, vb, bar);
-                }
-#pragma unroll
-                for (int i = 0; i < kStages; ++i) if (i == s) f[i].first = first;
+    auto issue = [&](int s, bool reuse) -> InFlight {   // bring position x_issue into stage s
+        InFlight f{0, 0u, 0u};
+        if (x_issue >= x_hi) return f;
+        if (x_issue - win_base >= 32) { win_base = x_issue; fill_window(win_base); }
+        const int src = (int)(x_issue - win_base);
+        const int page = __shfl_sync(0xFFFFFFFFu, win.page, src);
+        const int nv = __shfl_sync(0xFFFFFFFFu, win.n_valid, src);
+        const uint32_t first = __shfl_sync(0xFFFFFFFFu, win.first, src);
+        const uint32_t groups = __shfl_sync(0xFFFFFFFFu, win.groups, src);
+        if (page >= 0) {
+            const size_t row0 = (size_t)p_issue * a.T + (size_t)page * kPage;
+            if (lane < nv) f.mask = a.v_mask[row0 + lane];
+            f.nv = nv;
+            f.chunks = groups * OPG;
+            if (lane == 0) {
+                const uint32_t kb = (uint32_t)nv * kRowBytes, vb = groups * kGroupBytes;
+                const uint32_t bar = bars + 8 * s, dst = ring + (uint32_t)s * kStageBytes;
+                if (reuse) fence_proxy_async();  // the stage's earlier reads precede the new writes
+                mbar_expect_tx(bar, kb + vb);
+                bulk_g2s(dst, a.k + row0 * kRowBytes, kb, bar);
+                if (vb)
+                    bulk_g2s(dst + kKeyBytes,
+                             a.v_packed + ((size_t)p_issue * a.cap_groups + first) * kGroupBytes, vb, bar);
             }
-            ++x_issue;
-            if (++slot_issue == mp) { slot_issue = 0; ++p_issue; }
         }
-#pragma unroll
-        for (int i = 0; i < kStages; ++i) if (i == s) { f[i].nv = nv; f[i].chunks = chunks; }
+        ++x_issue;
+        if (++slot_issue == mp) { slot_issue = 0; ++p_issue; }
+        return f;
     };
 
     // ---- query operand ----------------------------------------------------------------------
@@ -269,8 +246,15 @@ decode_attn_kernel(const AttnArgs a) {
     auto compute = [&](int s, const InFlight& f) {
         const uint32_t kst = ring + (uint32_t)s * kStageBytes, vst = kst + kKeyBytes;
         const int nv = f.nv;
-        // groups of the page before this lane's token (offsets past the store are clipped like `first`)
-        const uint32_t pre = (uint32_t)min((long long)f.pre, (long long)a.cap_groups) - f.first;
+        // exclusive prefix (in groups) of the page's token masks, lanes 0..15
+        const uint32_t cnt = __popc(f.mask);
+        uint32_t pre = cnt;
+#pragma unroll
+        for (int d = 1; d < 16; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, pre, d);
+            if (lane >= d) pre += o;
+        }
+        pre -= cnt;
 
         if constexpr (MMA) {
             // S^T = K . Q^T : rows = tokens (r, r+8), columns = heads (2c, 2c+1)
@@ -288,27 +272,19 @@ decode_attn_kernel(const AttnArgs a) {
             sv[1] = v0 ? (s0[1] + s1[1]) * a.scale_log2 : -INFINITY;
             sv[2] = v1 ? (s0[2] + s1[2]) * a.scale_log2 : -INFINITY;
             sv[3] = v1 ? (s0[3] + s1[3]) * a.scale_log2 : -INFINITY;
-            // the running maxima move only when some token of the page exceeds them (after the first pages of a
-            // range that is rare): the cross-lane maximum and the rescaling are skipped otherwise, which leaves
-            // every value exactly as it would be (the factor would be 1)
             float pm0 = fmaxf(sv[0], sv[2]), pm1 = fmaxf(sv[1], sv[3]);
-            const bool grown = __any_sync(0xFFFFFFFFu, pm0 > m_run[0] || pm1 > m_run[1]);
-            float al0 = 1.f, al1 = 1.f;
-            if (grown) {
 #pragma unroll
-                for (int d = 4; d < 32; d <<= 1) {
-                    pm0 = fmaxf(pm0, __shfl_xor_sync(0xFFFFFFFFu, pm0, d));
-                    pm1 = fmaxf(pm1, __shfl_xor_sync(0xFFFFFFFFu, pm1, d));
-                }
-                const float mn0 = fmaxf(m_run[0], pm0), mn1 = fmaxf(m_run[1], pm1);   // finite: token 0 is valid
-                al0 = exp2f(m_run[0] - mn0); al1 = exp2f(m_run[1] - mn1);
-                m_run[0] = mn0; m_run[1] = mn1;
+            for (int d = 4; d < 32; d <<= 1) {
+                pm0 = fmaxf(pm0, __shfl_xor_sync(0xFFFFFFFFu, pm0, d));
+                pm1 = fmaxf(pm1, __shfl_xor_sync(0xFFFFFFFFu, pm1, d));
             }
-            const float mn0 = m_run[0], mn1 = m_run[1];
+            const float mn0 = fmaxf(m_run[0], pm0), mn1 = fmaxf(m_run[1], pm1);   // finite: token 0 is valid
+            const float al0 = exp2f(m_run[0] - mn0), al1 = exp2f(m_run[1] - mn1);
             const float p0 = exp2f(sv[0] - mn0), p1 = exp2f(sv[1] - mn1);
             const float p2 = exp2f(sv[2] - mn0), p3 = exp2f(sv[3] - mn1);
             l_run[0] = fmaf(l_run[0], al0, p0 + p2);
             l_run[1] = fmaf(l_run[1], al1, p1 + p3);
+            m_run[0] = mn0; m_run[1] = mn1;
             // P^T as B fragments: high bf16 part and bf16 residual
             const uint32_t wh0 = pack_bf16(p0, p1), wh1 = pack_bf16(p2, p3);
             const uint32_t wl0 = pack_bf16(p0 - bf16lo(wh0), p1 - bf16hi(wh0));
@@ -327,7 +303,7 @@ decode_attn_kernel(const AttnArgs a) {
                 const bool kept = ((m >> grp) & 1u) && idx < limit;
                 uint32_t a0, a1, a2, a3;
                 ldmatrix_x4_trans(kept ? vst + idx * 16u : zero_row, a0, a1, a2, a3);
-                if (grown) { acc[dt][0] *= al0; acc[dt][1] *= al1; acc[dt][2] *= al0; acc[dt][3] *= al1; }
+                acc[dt][0] *= al0; acc[dt][1] *= al1; acc[dt][2] *= al0; acc[dt][3] *= al1;
                 mma_bf16(acc[dt], a0, a1, a2, a3, bh0, bh1);
                 mma_bf16(acc[dt], a0, a1, a2, a3, bl0, bl1);
             }
@@ -360,18 +336,13 @@ decode_attn_kernel(const AttnArgs a) {
                 sd[hf] = (r + 8 * hf < nv) ? d * a.scale_log2 : -INFINITY;
             }
             float pm = fmaxf(sd[0], sd[1]);
-            const bool grown = __any_sync(0xFFFFFFFFu, pm > m_run[0]);   // else the maximum stays and the factor is 1
-            float al = 1.f;
-            if (grown) {
 #pragma unroll
-                for (int d = 4; d < 32; d <<= 1) pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, d));
-                const float mx = fmaxf(m_run[0], pm);
-                al = exp2f(m_run[0] - mx);
-                m_run[0] = mx;
-            }
-            const float mn = m_run[0];
+            for (int d = 4; d < 32; d <<= 1) pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, d));
+            const float mn = fmaxf(m_run[0], pm);
+            const float al = exp2f(m_run[0] - mn);
             const float p0 = exp2f(sd[0] - mn), p1 = exp2f(sd[1] - mn);
             l_run[0] = fmaf(l_run[0], al, p0 + p1);
+            m_run[0] = mn;
             const uint32_t limit = f.chunks;
             uint4 vr[2][4];
 #pragma unroll
@@ -549,8 +520,9 @@ decode_attn_kernel(const AttnArgs a) {
     };
 
     // ---- main loop ----------------------------------------------------------------------------
+    InFlight f[kStages];                          // f[0] = oldest page in flight, in stage s
 #pragma unroll
-    for (int i = 0; i < kStages; ++i) issue(i);
+    for (int i = 0; i < kStages; ++i) f[i] = issue(i, false);
 
     int p_cur = (int)(x_lo / mp);
     int slot_cur = (int)(x_lo - (long long)p_cur * mp);
@@ -560,10 +532,7 @@ decode_attn_kernel(const AttnArgs a) {
     int s = 0;
 #pragma unroll 1
     for (int n = 0; n < count; ++n) {
-        InFlight cur{0, 0u, 0u, 0u, 0u};
-#pragma unroll
-        for (int i = 0; i < kStages; ++i) if (i == s) cur = f[i];
-        if (cur.nv > 0) {                         // uniform across the warp
+        if (f[0].nv > 0) {                        // uniform across the warp
             const uint32_t par = (phase >> s) & 1u;
             phase ^= 1u << s;
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(bars + 8 * s, par))) {
@@ -571,15 +540,20 @@ decode_attn_kernel(const AttnArgs a) {
                 // one more bounded wait each so they do not land in a dead CTA's memory,
                 // and leave; the outputs this worker owes stay unwritten.
                 if (lane == 0) atomicExch(a.status, (int)STC_ERR_TIMEOUT);
+                int s2 = s;
 #pragma unroll
-                for (int i = 0; i < kStages; ++i)
-                    if (i != s && f[i].nv > 0) mbar_wait(bars + 8 * i, (phase >> i) & 1u);
+                for (int i = 1; i < kStages; ++i) {
+                    s2 = s2 + 1 == kStages ? 0 : s2 + 1;
+                    if (f[i].nv > 0) mbar_wait(bars + 8 * s2, (phase >> s2) & 1u);
+                }
                 return;
             }
-            compute(s, cur);
+            compute(s, f[0]);
         }
         __syncwarp();
-        issue(s);
+#pragma unroll
+        for (int i = 0; i + 1 < kStages; ++i) f[i] = f[i + 1];
+        f[kStages - 1] = issue(s, true);
         s = s + 1 == kStages ? 0 : s + 1;
         ++slot_cur;
         if (slot_cur == mp || n + 1 == count) {   // the range leaves this problem (one call site: finish is big)
@@ -695,9 +669,10 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
     }
 #undef STC_ATTN_LAUNCH
 #undef STC_ATTN
-    return e != cudaSuccess ? e : cudaGetLastError();
+    return cudaGetLastError();
 }
 
+// status word + page counters of a call
 cudaError_t clear_decode_attn_ws(const Geom& g, void* ws, cudaStream_t st) {
     return cudaMemsetAsync(ws, 0, 256 + (size_t)g.problems * 4, st);
 }
