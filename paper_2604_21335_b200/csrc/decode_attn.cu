@@ -579,15 +579,20 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // Workers (warps) and partial slots per problem.  Sized from max_pages only, so the
 // workspace query and the launch agree; independent of the device so that the
 // workspace size can be asked for without one.
+// The plan is sized for kPlanSms multiprocessors: the workspace size has to be computable without a
+// device (stc_workspace_bytes is host arithmetic), so the plan uses the B200's count as a documented
+// constant; the launch only picks the ring depth from the device it runs on.
+constexpr long long kPlanSms = 148;
+
 AttnPlan attn_plan(const Geom& g, int max_pages) {
     AttnPlan p;
     const long long mp = max_pages < 1 ? 1 : max_pages;
     const long long total = (long long)(g.problems < 1 ? 1 : g.problems) * mp;
     long long workers = (total + kMinPagesPerWarp - 1) / kMinPagesPerWarp;
-    const long long wave = 148LL * kCtasPerSm * kWarps;
+    const long long wave = kPlanSms * kCtasPerSm * kWarps;
     if (workers > wave) workers = wave;
     // a call that fits one CTA per SM runs there, with the deeper ring
-    if (workers > 148LL * kWarps && workers < 148LL * kWarps * 3 / 2) workers = 148LL * kWarps;
+    if (workers > kPlanSms * kWarps && workers < kPlanSms * kWarps * 3 / 2) workers = kPlanSms * kWarps;
     // many short problems: one warp per problem, so that no problem is split and nothing is merged
     if (g.problems <= wave && 2LL * g.problems >= workers) workers = g.problems;
     const long long by_slots = (long long)(kMaxSlots - 1) * (g.problems < 1 ? 1 : g.problems);
@@ -649,7 +654,10 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
     if (!(flags & kLaunchNoClear)) e = clear_decode_attn_ws(g, ws, st);
     if (e != cudaSuccess) return e;
     const int n_cta = (p.n_workers + kWarps - 1) / kWarps;
-    const bool mma = g.Gq > 1, deep = n_cta <= 148;
+    int sms = 0;
+    e = device_sm_count(&sms);
+    if (e != cudaSuccess) return e;
+    const bool mma = g.Gq > 1, deep = n_cta <= sms;      // a call that fits one CTA per SM takes the deeper ring
 #define STC_ATTN_LAUNCH(S_, MMA_, ST_)                                                                  \
     do {                                                                                                \
         cudaFuncSetAttribute(decode_attn_kernel<S_, MMA_, ST_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \

@@ -727,18 +727,25 @@ namespace {
 // CTAs of the select kernel that can be resident at once (it is launched cooperatively).
 template <int S>
 cudaError_t select_grid_limit(int* limit) {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, sms = 0, per_sm = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // per device: the occupancy of the kernel is a property of the kernel and the device, the
+    // query is cheap next to a cooperative launch, and a process may drive several devices
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cached[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    int v = (dev >= 0 && dev < kMaxDevices) ? cached[dev].load() : 0;
+    if (v == 0) {
+        int sms = 0, per_sm = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, route_select_kernel<S>, kThreads, 0);
         if (e != cudaSuccess) return e;
         if (sms <= 0 || per_sm <= 0) return cudaErrorLaunchOutOfResources;
-        cached = sms * per_sm;
+        v = sms * per_sm;
+        if (dev >= 0 && dev < kMaxDevices) cached[dev].store(v);
     }
-    *limit = cached;
+    *limit = v;
     return cudaSuccess;
 }
 
@@ -786,7 +793,10 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
         e = cudaMemsetAsync(w.state, 0, small ? w.zero_small : w.zero_bytes, st);
         if (e != cudaSuccess) return e;
     }
-    const unsigned grid_small = (unsigned)(g.problems < 148 * 16 ? g.problems : 148 * 16);
+    int sms = 0;
+    e = device_sm_count(&sms);
+    if (e != cudaSuccess) return e;
+    const unsigned grid_small = (unsigned)(g.problems < sms * 16 ? g.problems : sms * 16);
 
 #define STC_ROUTE(S_)                                                                               \
     case S_: {                                                                                      \
