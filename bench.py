@@ -630,10 +630,10 @@ KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kern
 # kernel from the committed ncu captures under profiles/, keyed by (workload, batch, budget, keep, call);
 # absent = no capture of the kernel as it stands.
 TRAFFIC_NOTE: dict = {
-    # quest_filter_kernel<4>: dram__bytes_read 134.62 MB + dram__bytes_write 4.01 MB per launch at batch 4
+    # quest_filter_kernel<4>: dram__bytes_read 134.71 MB + dram__bytes_write 4.36 MB per launch at batch 4
     # (profiles/ncu_full_select_attn_cfg4_batch4.md), scaled by 4 to the 16 sequences of the full workload (the
     # traffic is the metadata scan plus the score array, both proportional to the number of problems)
-    ("cfg4", 16, 4096, 4, "quest_select"): 4 * (134.62e6 + 4.01e6),
+    ("cfg4", 16, 4096, 4, "quest_select"): 4 * (134.71e6 + 4.36e6),
 }
 
 
