@@ -16,8 +16,10 @@
 // Lane 0 brings both in with two bulk asynchronous copies (cp.async.bulk, the 1-D
 // TMA path) that signal the stage's mbarrier; the copies for the next kStages-1
 // pages are in flight while the warp computes on the current one, which is what
-// hides HBM latency (3 stages at 8 warps per SM; 6 stages at 4 warps per SM when
-// the call is too small to fill a wave and per-warp latency is what counts).  The list entry, sequence length and value
+// hides HBM latency (3 stages at 8 warps per SM; 6 stages at 4 warps per SM when the call is too
+// small to fill a wave and per-warp latency is what counts; 2 stages at 12 warps per SM for
+// the single-head path on full-size calls, where a warp's per-page arithmetic is longer than a
+// copy's latency and more warps buy more than a deeper ring).  The list entry, sequence length and value
 // offsets a copy needs are fetched 32 pages at a time, one page per lane.
 //
 // A dropped value group is never copied for its own sake and never read: the
@@ -48,6 +50,9 @@ constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kStagesWide = 3;                   // two CTAs per SM (full-size calls)
 constexpr int kStagesDeep = 6;                   // one CTA per SM (calls too small to fill a wave)
+constexpr int kStagesLean = 2;                   // three CTAs per SM: the single-head path on full-size calls, whose
+                                                 // per-page arithmetic (not the copies) sets the pace, so that
+                                                 // twelve warps per SM beat eight with a deeper ring
 constexpr int kMaxGq = 8;
 constexpr int kCtasPerSm = 2;
 constexpr int kMinPagesPerWarp = 4;
@@ -120,7 +125,7 @@ struct PageRef {
 };
 
 template <int S, bool MMA, int kStages>
-__global__ void __launch_bounds__(kThreads, kStages == kStagesWide ? kCtasPerSm : 1)
+__global__ void __launch_bounds__(kThreads, kStages == kStagesLean ? 3 : (kStages == kStagesWide ? kCtasPerSm : 1))
 decode_attn_kernel(const AttnArgs a) {
     constexpr uint32_t kRingBytes = ring_bytes(kStages);
     constexpr int OPG = kOctets / S;             // 16-byte chunks per value group
@@ -589,12 +594,14 @@ AttnPlan attn_plan(const Geom& g, int max_pages) {
     const long long mp = max_pages < 1 ? 1 : max_pages;
     const long long total = (long long)(g.problems < 1 ? 1 : g.problems) * mp;
     long long workers = (total + kMinPagesPerWarp - 1) / kMinPagesPerWarp;
-    const long long wave = kPlanSms * kCtasPerSm * kWarps;
+    const long long wave = kPlanSms * (g.Gq == 1 ? 3 : kCtasPerSm) * kWarps;   // resident warps (see kStagesLean)
     if (workers > wave) workers = wave;
     // a call that fits one CTA per SM runs there, with the deeper ring
     if (workers > kPlanSms * kWarps && workers < kPlanSms * kWarps * 3 / 2) workers = kPlanSms * kWarps;
-    // many short problems: one warp per problem, so that no problem is split and nothing is merged
-    if (g.problems <= wave && 2LL * g.problems >= workers) workers = g.problems;
+    // many short problems: one warp per problem, so that no problem is split and nothing is merged (long
+    // single-head problems that would leave a third of the warps idle are split all the same)
+    if (g.problems <= wave && 2LL * g.problems >= workers && !(g.Gq == 1 && mp >= 64 && 10LL * g.problems < 7 * wave))
+        workers = g.problems;
     const long long by_slots = (long long)(kMaxSlots - 1) * (g.problems < 1 ? 1 : g.problems);
     if (workers > by_slots) workers = by_slots;  // keeps ceil(workers / problems) + 1 <= kMaxSlots
     if (workers < 1) workers = 1;
@@ -669,6 +676,7 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
         if (mma && deep) STC_ATTN_LAUNCH(S_, true, kStagesDeep);                                        \
         else if (mma) STC_ATTN_LAUNCH(S_, true, kStagesWide);                                           \
         else if (deep) STC_ATTN_LAUNCH(S_, false, kStagesDeep);                                         \
+        else if (n_cta > 2 * sms) STC_ATTN_LAUNCH(S_, false, kStagesLean);                              \
         else STC_ATTN_LAUNCH(S_, false, kStagesWide);                                                   \
         break;
     switch (g.S) {
