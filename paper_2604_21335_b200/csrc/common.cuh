@@ -162,6 +162,9 @@ cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kma
                                 int token_budget, int n_recent_pages, int max_pages, int32_t* page_ids,
                                 int32_t* n_pages, float* scores_opt, void* ws, cudaStream_t st, unsigned flags = 0);
 cudaError_t clear_quest_select_ws(const Geom& g, void* ws, cudaStream_t st);
+size_t quest_select_clear_bytes(const Geom& g);    // leading bytes of the workspace a call needs zeroed
+// One small kernel that zeroes the leading bytes of two workspaces (one graph node instead of two memsets).
+cudaError_t clear_two(void* a, size_t a_bytes, void* b, size_t b_bytes, cudaStream_t st);
 
 cudaError_t launch_pages_to_class(const Geom& g, const int32_t* page_ids, const int32_t* n_pages,
                                   int max_pages, uint8_t* tok_class, cudaStream_t st);
@@ -200,5 +203,6 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
                                int max_pages, float sm_scale, float* out, float* lse, void* ws,
                                cudaStream_t st, unsigned flags = 0);
 cudaError_t clear_decode_attn_ws(const Geom& g, void* ws, cudaStream_t st);
+size_t decode_attn_clear_bytes(const Geom& g);     // leading bytes of the workspace a call needs zeroed
 
 }  // namespace stc

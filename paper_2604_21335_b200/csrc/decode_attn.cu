@@ -689,8 +689,10 @@ cudaError_t launch_decode_attn(const Geom& g, const void* k, const void* v_packe
 }
 
 // status word + page counters of a call
+size_t decode_attn_clear_bytes(const Geom& g) { return 256 + (size_t)g.problems * 4; }
+
 cudaError_t clear_decode_attn_ws(const Geom& g, void* ws, cudaStream_t st) {
-    return cudaMemsetAsync(ws, 0, 256 + (size_t)g.problems * 4, st);
+    return cudaMemsetAsync(ws, 0, decode_attn_clear_bytes(g), st);
 }
 
 }  // namespace stc

@@ -1113,8 +1113,27 @@ size_t select_ws_bytes(const Geom& g) {
     return 256 + counters_bytes(g) + (size_t)g.problems * g.P * sizeof(float);
 }
 
+size_t quest_select_clear_bytes(const Geom& g) { return 256 + (size_t)g.problems * 16; }
+
 cudaError_t clear_quest_select_ws(const Geom& g, void* ws, cudaStream_t st) {
-    return cudaMemsetAsync(ws, 0, 256 + (size_t)g.problems * 16, st);
+    return cudaMemsetAsync(ws, 0, quest_select_clear_bytes(g), st);
+}
+
+namespace {
+__global__ void clear_two_kernel(uint4* a, size_t na, uint4* b, size_t nb) {     // counts in 16-byte words
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < na + nb; i += (size_t)gridDim.x * blockDim.x)
+        if (i < na) a[i] = z; else b[i - na] = z;
+}
+}  // namespace
+
+cudaError_t clear_two(void* a, size_t a_bytes, void* b, size_t b_bytes, cudaStream_t st) {
+    // both ranges start on 256-byte boundaries and are rounded up to 16 bytes (the words behind them are
+    // score / partial storage that the call rewrites anyway)
+    const size_t na = (a_bytes + 15) / 16, nb = (b_bytes + 15) / 16;
+    const unsigned blocks = (unsigned)((na + nb + 255) / 256 < 64 ? (na + nb + 255) / 256 : 64);
+    clear_two_kernel<<<blocks ? blocks : 1, 256, 0, st>>>(static_cast<uint4*>(a), na, static_cast<uint4*>(b), nb);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_quest_select(const Geom& g, const void* kmin, const void* kmax, const void* q,

@@ -308,8 +308,7 @@ int32_t stc_decode_step(const stc_shape* shape, const stc_cache* cache, const vo
     if (rc != STC_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // both workspaces are cleared first, so that nothing stands between the two kernels
-    cudaError_t e = clear_quest_select_ws(g, ws_select, st);
-    if (e == cudaSuccess) e = clear_decode_attn_ws(g, ws_attn, st);
+    cudaError_t e = clear_two(ws_select, quest_select_clear_bytes(g), ws_attn, decode_attn_clear_bytes(g), st);
     if (e == cudaSuccess)
         e = launch_quest_select(g, cache->kmin, cache->kmax, q, token_budget, 0, max_pages, page_ids, n_pages,
                                 nullptr, ws_select, st, kLaunchNoClear);
