@@ -487,7 +487,7 @@ static_assert(kFSmemBytes <= 227 * 1024 - 2048, "ring + selection scratch fit on
 //      k-th key, and counts, per warp, the keys in the bins above them;
 //   C. the k-th largest key t is ranked among the candidates; candidates above t + 2 delta are
 //      selected, those below t - 2 delta are not, the rest are scored exactly and ranked by
-//      (exact score descending, page ascending); the verdicts are written into the staged keys;
+//      (exact score descending, page ascending); the decisions are written into the staged keys;
 //   D. one pass writes the selected pages in ascending order (ballot ranks inside a warp's
 //      contiguous block, block offsets from the per-warp counts).
 template <int NT>
@@ -622,7 +622,7 @@ __device__ __noinline__ bool filter_select_fast(const float* __restrict__ u, int
         asm volatile("prefetch.global.L2 [%0];" ::"l"(row + 128 * (e & 1)));
     }
 
-    // ---- C. the k-th largest approximate key, then the verdict on every candidate -----------------
+    // ---- C. the k-th largest approximate key, then the decision on every candidate -----------------
     for (int e = tid; e < ncand; e += NT) {
         const uint32_t x = ckey[e];
         if ((int)((x >> shift) & dmask) != bin) continue;

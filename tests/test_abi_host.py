@@ -104,3 +104,30 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(Bd, "_LIB_PATH", tmp_path / "libstc.so")
     with pytest.raises(ImportError):
         Bd.load_library()
+
+
+def test_newer_calls_reject_bad_arguments_before_any_launch(lib):
+    cs = shape().c()
+    cc = Bd._Cache()
+    st = None
+    fake = C.c_void_p(0x1000)
+    full = Bd._Cache(fake, fake, fake, fake, fake, fake, 100)
+    # stc_decode_step: null cache pointers, list stride below the budget's page count, workspaces missing
+    assert lib.stc_decode_step(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, 0.1, fake, None, fake, 1 << 30,
+                               fake, 1 << 30, st) == 1
+    assert lib.stc_decode_step(C.byref(cs), C.byref(full), fake, 1024, 63, fake, fake, 0.1, fake, None, fake, 1 << 30,
+                               fake, 1 << 30, st) == 1
+    assert lib.stc_decode_step(C.byref(cs), C.byref(full), fake, 1024, 64, fake, fake, 0.1, fake, None, None, 0,
+                               fake, 1 << 30, st) == 3
+    assert lib.stc_decode_step(C.byref(cs), C.byref(full), fake, 1024, 64, fake, fake, 0.1, fake, None, fake, 1 << 30,
+                               fake, 16, st) == 3
+    # stc_route_new_pages: budget above S, bad mode, null scores
+    assert lib.stc_route_new_pages(C.byref(cs), C.byref(full), fake, fake, 9, 1, 0, fake, fake, st) == 1
+    assert lib.stc_route_new_pages(C.byref(cs), C.byref(full), fake, fake, 4, 1, 7, fake, fake, st) == 1
+    assert lib.stc_route_new_pages(C.byref(cs), C.byref(full), None, fake, 4, 1, 0, fake, fake, st) == 1
+    # stc_pages_to_class: null output
+    assert lib.stc_pages_to_class(C.byref(cs), fake, fake, 64, None, st) == 1
+    # stc_decode_step_host: arena too small
+    out = C.c_size_t(0)
+    assert lib.stc_decode_step_host_arena_bytes(C.byref(cs), 1024, C.byref(out)) == 0 and out.value > 0
+    assert lib.stc_decode_step_host(C.byref(cs), C.byref(full), fake, 1024, 0.1, fake, 16, fake, fake, st) == 3
