@@ -39,15 +39,25 @@ constexpr int kTokPerThread = kTile / kThreads;
 constexpr int kBins = 2048;
 
 // state words per problem
-enum { ST_NROUTED = 0, ST_PREFIX, ST_KREM, ST_FLAGS, ST_TICKET0, ST_TICKET1, ST_TICKET2, ST_DONE, ST_WORDS };
+enum { ST_NROUTED = 0, ST_PREFIX, ST_KREM, ST_FLAGS, ST_TICKET0, ST_TICKET1, ST_TICKET2, ST_DONE,
+       // words of the band kernel (it leaves the eight above to the multi-pass kernel, except the results
+       // ST_KREM / ST_FLAGS / ST_PREFIX that the compaction reads)
+       ST_PATH, ST_BLO, ST_BHI, ST_LISTN, ST_TICKETA, ST_TICKETB, ST_DONEA, ST_NROUTEDA, ST_NROUTEDB, ST_ABOVE,
+       ST_SPARE0, ST_SPARE1, ST_WORDS };
 enum { FL_NONE = 1, FL_BUDGET = 2 };          // nothing beyond the reserved groups / budget error
+enum { PATH_OPEN = 0, PATH_BAND = 1, PATH_WIDE = 2 };   // who settles the problem: nobody yet / band kernel / multi-pass kernel
 // ST_DONE = histogram passes resolved so far (3 = threshold final)
+constexpr int kBins13 = 8192;                 // first digit of the band kernel: the top 13 key bits
+constexpr int kShift13 = 19;
 
 struct RouteWs {
     uint32_t* state;      // [problems][ST_WORDS]
     uint32_t* hist;       // [problems][3][kBins]
-    uint32_t* abort_word; // set when a bounded wait gave up
-    uint32_t* unit_sums;  // [problems][units]: definite count | tie count << 16
+    uint32_t* hist13;     // [problems][kBins13]
+    uint32_t* abort_word; // set when a bounded wait gave up; the next word: some problem is left to the multi-pass kernel
+    uint2* list;          // [problems][list_cap] (key, flat index) of the candidates in the threshold's bin
+    uint32_t list_cap;
+    uint32_t* unit_sums;  // [problems][units]: definite count | tie count << 16 (the band kernel adds to zeroed words)
     uint16_t* tie;        // [problems][T]
     size_t zero_small;    // leading bytes cleared per call: state and abort word only ...
     size_t zero_bytes;    // ... or with the global histograms (problems that span several CTAs)
@@ -65,9 +75,15 @@ RouteWs carve(const Geom& g, void* ws) {
     r.abort_word = reinterpret_cast<uint32_t*>(p + o); o += 256;
     r.zero_small = o;
     r.hist = reinterpret_cast<uint32_t*>(p + o);  o += align256((size_t)g.problems * 3 * kBins * 4);
-    r.zero_bytes = o;
+    const bool small = n_units <= 32 / g.S;       // (the one-CTA-per-problem kernel needs neither of the next two)
+    r.hist13 = reinterpret_cast<uint32_t*>(p + o); o += small ? 0 : align256((size_t)g.problems * kBins13 * 4);
     r.unit_sums = reinterpret_cast<uint32_t*>(p + o); o += align256((size_t)g.problems * n_units * 4);
+    r.zero_bytes = o;
     r.tie = reinterpret_cast<uint16_t*>(p + o);   o += align256((size_t)g.problems * g.T * 2);
+    // a sixteenth of a problem's keys (one bin of the 13-bit digit holds a few per cent at most on smooth data)
+    const size_t cap = small ? 0 : (((size_t)g.T * g.S / 16 + 4095) & ~(size_t)4095);
+    r.list_cap = (uint32_t)(cap < 0x40000000u ? cap : 0x40000000u);
+    r.list = reinterpret_cast<uint2*>(p + o);     o += align256((size_t)g.problems * r.list_cap * sizeof(uint2));
     r.total_bytes = o;
     return r;
 }
@@ -324,8 +340,10 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
                     uint32_t* __restrict__ hist_all, uint32_t* __restrict__ abort_word,
                     uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
                     uint32_t* __restrict__ unit_sums, long long total_units, int first_pass,
-                    unsigned long long wait_ns) {
+                    unsigned long long wait_ns, int only_wide) {
     constexpr int kBatch = 32 / S;               // tokens in flight per thread (32 score registers)
+    // after the band kernel: only the problems it left (PATH_WIDE) are this kernel's, usually none
+    if (only_wide && __ldcg(abort_word + 1) == 0u) return;
     __shared__ uint32_t shist[kBins];
     __shared__ uint32_t s_w[kWarps];
     __shared__ uint32_t s_red[kBatch][kWarps];
@@ -352,6 +370,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             const int b = problem / Hkv, hk = problem - b * Hkv;
             const int len = clamp_len(seq_len, b, T);
             uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+            if (only_wide && __ldcg(state + ST_PATH) != PATH_WIDE) continue;
             uint32_t* hist = hist_all + ((size_t)problem * 3 + pass) * kBins;
             const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
             uint4 raw[kBatch][S / 4];
@@ -453,6 +472,7 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
         x += n;
         const int b = problem / Hkv, hk = problem - b * Hkv;
         const int len = clamp_len(seq_len, b, T);
+        if (only_wide && __ldcg(state_all + (size_t)problem * ST_WORDS + ST_PATH) != PATH_WIDE) continue;
         const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
         uint4 raw[kBatch][S / 4];
         int cls_of[kBatch];
@@ -507,6 +527,532 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
             __syncthreads();
         }
     }
+}
+
+// ---- the band kernel -----------------------------------------------------------------------
+// One scan of the scores (and a fraction of another) instead of four.
+//   Scan A looks at a sample of every problem (runs of four consecutive tokens, evenly spread; all
+//   tokens when the problem is small) and histograms the top 13 key bits of the sample's candidates.
+//   The CTA that completes a problem's sample derives a BAND of bins that holds the take-th largest
+//   candidate of the whole problem with near certainty: the bins of the sample ranks
+//   f m -+ (5 sqrt(m f (1 - f)) + 2), f = take / candidates = (K - floor) / (S - floor), m = sample size.
+//   Scan B reads every score once: candidates above the band are kept (their definite bits are
+//   written straight away and counted), those below are dropped, those inside -- a per cent or two
+//   of the problem -- are appended as (key, flat index) pairs to the problem's list.  All tests are
+//   float comparisons against the band's two edges; keys are only built for the list.
+//   The CTA that completes scan B of a problem settles it exactly: with `above` pairs counted above
+//   the band, the take-th largest candidate is the (take - above)-th largest of the list, provided
+//   above < take <= above + list length -- which is the check that the band was right.  Radix select
+//   over the list (three passes, the list sits in L2), then one pass that sets the definite bit of
+//   every listed pair above the threshold and the tie bit of every pair on it (the compaction
+//   resolves ties in flat-index order, as after the multi-pass kernel).
+// A problem whose band was wrong, or holds more pairs than the list has room for (massive ties), is
+// marked PATH_WIDE and left to the multi-pass kernel that runs next; the result is the same either way.
+
+template <bool kSharedHist>
+__device__ void pick_digit_n(const uint32_t* __restrict__ hist, int nbins, int per, uint32_t krem,
+                             uint32_t* s_w, uint32_t* s_out /*[3]*/) {
+    const int top = nbins - 1 - per * (int)threadIdx.x;
+    uint32_t sum = 0;
+    // a histogram in global memory: the thread's bins are `per` consecutive words ending at `top`, read as
+    // 16-byte pieces that are all in flight together (per = 32, nbins = per * kThreads)
+    constexpr int kQuads = 8;
+    const bool quads = !kSharedHist && per == 4 * kQuads && top - per + 1 >= 0;
+    uint32_t qsum[kQuads];
+    if (quads) {
+        const uint4* h4 = reinterpret_cast<const uint4*>(hist + top - per + 1);
+#pragma unroll
+        for (int j = 0; j < kQuads; ++j) {
+            const uint4 v = __ldcg(h4 + j);
+            qsum[j] = v.x + v.y + v.z + v.w;
+            sum += qsum[j];
+        }
+    } else {
+#pragma unroll 4
+        for (int j = 0; j < per; ++j) {
+            const int bin = top - j;
+            sum += bin >= 0 ? (kSharedHist ? hist[bin] : __ldcg(hist + bin)) : 0u;
+        }
+    }
+    const uint32_t excl = block_excl_scan(sum, s_w, nullptr);
+    if (excl < krem && krem <= excl + sum) {
+        uint32_t run = excl;
+        int j0 = 0, j1 = per;
+        if (quads) {                                // first the piece (from the top one down), then the bin inside it
+            int piece = 0;
+            bool found = false;
+#pragma unroll
+            for (int q = kQuads - 1; q >= 0; --q) {
+                if (!found) {
+                    if (run + qsum[q] >= krem) { piece = q; found = true; }
+                    else run += qsum[q];
+                }
+            }
+            j0 = (kQuads - 1 - piece) * 4;
+            j1 = j0 + 4;
+        }
+        for (int j = j0; j < j1; ++j) {
+            const int bin = top - j;
+            const uint32_t c = bin >= 0 ? (kSharedHist ? hist[bin] : __ldcg(hist + bin)) : 0u;
+            if (run + c >= krem) {
+                s_out[0] = (uint32_t)bin;
+                s_out[1] = krem - run;
+                s_out[2] = c;
+                break;
+            }
+            run += c;
+        }
+    }
+    __syncthreads();
+}
+
+// Sets bits of a 16-bit mask word that other threads may be updating.  word_ok: the mask array starts
+// on a 4-byte boundary and a problem's masks never share a 32-bit word with another problem's, so the
+// update can be a 32-bit reduction (nothing comes back, nothing waits); otherwise a 16-bit
+// compare-and-swap loop.
+__device__ __forceinline__ void or16(uint16_t* p, uint32_t bits, bool word_ok) {
+    if (word_ok) {
+        const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+        atomicOr(reinterpret_cast<unsigned int*>(a & ~(uintptr_t)3), bits << ((a & 2) ? 16 : 0));
+    } else {
+        unsigned short* q = reinterpret_cast<unsigned short*>(p);
+        unsigned short old = *reinterpret_cast<volatile unsigned short*>(q), assumed;
+        do {
+            assumed = old;
+            old = atomicCAS(q, assumed, (unsigned short)(assumed | bits));
+        } while (old != assumed);
+    }
+}
+
+// Wait (bounded) until the problem's band is published, then broadcast it: s_bc = {ok, path, b_lo, b_hi}.
+__device__ __forceinline__ bool wait_band(const uint32_t* state, uint32_t* s_bc, uint32_t* abort_word,
+                                          uint64_t wait_ns) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t ok = 1;
+        if (ld_acquire(state + ST_DONEA) == 0u) {
+            const uint64_t t0 = globaltimer_ns();
+            while (ld_acquire(state + ST_DONEA) == 0u) {
+                __nanosleep(100);
+                if (globaltimer_ns() - t0 > wait_ns || ld_acquire(abort_word) != 0u) { ok = 0; break; }
+            }
+        }
+        if (!ok) atomicExch(abort_word, 1u);
+        s_bc[0] = ok;
+        s_bc[1] = __ldcg(state + ST_PATH);
+        s_bc[2] = __ldcg(state + ST_BLO);
+        s_bc[3] = __ldcg(state + ST_BHI);
+    }
+    __syncthreads();
+    return s_bc[0] != 0u;
+}
+
+// The scores whose 13-bit digit lies in [b_lo, b_hi], as a closed float interval (scores are not NaN).
+__device__ __forceinline__ void band_bounds(uint32_t b_lo, uint32_t b_hi, float& lo, float& hi) {
+    uint32_t klo = b_lo << kShift13, khi = (b_hi << kShift13) | ((1u << kShift13) - 1u);
+    klo = max(klo, 0x007FFFFFu);                   // -inf
+    khi = min(khi, 0xFF800000u);                   // +inf
+    if (khi == 0x7FFFFFFFu) khi = 0x7FFFFFFEu;     // the key of -0 is unused: stop below zero
+    lo = key_float(klo);
+    hi = key_float(khi);
+}
+
+// Definite bits and list candidates of one routed token against the band, on the raw scores.  The scan is
+// bound by the integer / compare pipe, so the work per score is kept to two comparisons: one against each
+// edge (a candidate is at or above the lower edge and not above the upper one).  The reserved group -- the
+// token's first maximum -- only has to be looked for when no score lies above the band: otherwise the
+// maximum is above the band too, and it changes neither the definite bits nor the candidates.
+template <int S>
+__device__ __forceinline__ void band_token(const uint4 (&raw)[S / 4], bool select, float lo, float hi,
+                                           int min_per_token, uint32_t& def, uint32_t& cand) {
+    float x[S];
+#pragma unroll
+    for (int i = 0; i < S / 4; ++i) {
+        x[4 * i + 0] = __uint_as_float(raw[i].x);
+        x[4 * i + 1] = __uint_as_float(raw[i].y);
+        x[4 * i + 2] = __uint_as_float(raw[i].z);
+        x[4 * i + 3] = __uint_as_float(raw[i].w);
+    }
+    def = 0;
+    cand = 0;
+    if (select) {
+        uint32_t ge = 0;
+#pragma unroll
+        for (int j = 0; j < S; ++j) {
+            def |= (x[j] > hi ? 1u : 0u) << j;
+            ge |= (x[j] >= lo ? 1u : 0u) << j;
+        }
+        cand = ge & ~def;
+    }
+    if (min_per_token && def == 0u) {
+        float bx = x[0];
+        int best = 0;
+#pragma unroll
+        for (int j = 1; j < S; ++j) {
+            const bool up = x[j] > bx;             // (-0 and +0 compare equal here and as keys)
+            bx = up ? x[j] : bx;
+            best = up ? j : best;
+        }
+        def = 1u << best;
+        cand &= ~def;
+    }
+}
+
+// Key j of a token's raw scores (j known at run time: selected by value, no indexed registers).
+template <int S>
+__device__ __forceinline__ uint32_t raw_word(const uint4 (&raw)[S / 4], int j) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int i = 0; i < S / 4; ++i) {
+        w = j == 4 * i + 0 ? raw[i].x : w;
+        w = j == 4 * i + 1 ? raw[i].y : w;
+        w = j == 4 * i + 2 ? raw[i].z : w;
+        w = j == 4 * i + 3 ? raw[i].w : w;
+    }
+    return w;
+}
+
+// The list of a problem is complete: find the krem-th largest of its keys and set the bits.
+template <int S>
+__device__ __noinline__ void settle_band(const uint2* __restrict__ list, uint32_t n_list, uint32_t krem,
+                                         uint32_t* __restrict__ state, uint16_t* __restrict__ mask_row,
+                                         uint16_t* __restrict__ tie_row, uint32_t* __restrict__ sums_row,
+                                         bool word_ok, uint32_t* shist, uint32_t* s_w, uint32_t* s_pick) {
+    const int tid = threadIdx.x;
+    constexpr int kInFlight = 16;                   // list entries a thread has in flight (the list sits in L2)
+    uint32_t prefix = 0;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {          // 11 + 11 + 10 bits
+        const uint32_t himask = pass_himask(pass);
+        const int dshift = pass_shift(pass);
+        const int nbins = pass == 2 ? 1024 : 2048;
+        for (int i = tid; i < nbins; i += kThreads) shist[i] = 0u;
+        __syncthreads();
+#pragma unroll 1
+        for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kThreads) {
+            uint32_t k[kInFlight];
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i) k[i] = __ldcg(&list[min(e0 + i * kThreads, n_list - 1)].x);
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i)
+                if (e0 + i * kThreads < n_list && (k[i] & himask) == prefix)
+                    atomicAdd(&shist[(k[i] >> dshift) & (uint32_t)(nbins - 1)], 1u);
+        }
+        __syncthreads();
+        pick_digit_n<true>(shist, nbins, nbins / kThreads, krem, s_w, s_pick);
+        prefix |= s_pick[0] << dshift;
+        krem = s_pick[1];
+        __syncthreads();
+    }
+    const uint32_t tau = prefix;                    // krem: how many of the pairs on the threshold are kept
+#pragma unroll 1
+    for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kThreads) {
+        uint2 en[kInFlight];
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) en[i] = __ldcg(&list[min(e0 + i * kThreads, n_list - 1)]);
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) {
+            if (e0 + i * kThreads >= n_list || en[i].x < tau) continue;
+            const uint32_t t = en[i].y / S, j = en[i].y - t * S;
+            if (en[i].x > tau) {
+                or16(mask_row + t, 1u << j, word_ok);
+                atomicAdd(sums_row + t / kUnit, 1u);
+            } else {
+                or16(tie_row + t, 1u << j, word_ok);
+                atomicAdd(sums_row + t / kUnit, 1u << 16);
+            }
+        }
+    }
+    if (tid == 0) { state[ST_PREFIX] = tau; state[ST_KREM] = krem; }
+}
+
+// samp: 1, 2, 4 or 8 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
+// a standard deviation of the sample rank (50 in production).
+template <int S>
+__global__ void __launch_bounds__(kThreads, 4)
+route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
+                  int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int upp,
+                  int k_nominal, int min_per_token, uint32_t* __restrict__ state_all,
+                  uint32_t* __restrict__ hist_all, uint32_t* __restrict__ abort_word,
+                  uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
+                  uint32_t* __restrict__ unit_sums, uint2* __restrict__ list_all, uint32_t list_cap,
+                  long long total_units, int skip_scan_a, unsigned long long wait_ns, int samp, int z_tenths) {
+    constexpr int kBatch = S >= 8 ? 32 / S : 4;  // tokens in flight per thread (at most 32 score registers)
+    __shared__ uint32_t shist[kBins13];
+    __shared__ uint32_t s_w[kWarps];
+    __shared__ uint32_t s_pick[3];
+    __shared__ uint32_t s_bc[4];
+    __shared__ uint32_t s_cnt[2];
+    __shared__ int s_last;
+    constexpr int kStage = 64;                   // list entries a warp can hold back
+    __shared__ uint2 s_stage[kWarps][kStage];
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    uint2* stage = s_stage[tid >> 5];
+    const long long x0 = total_units * blockIdx.x / gridDim.x;
+    const long long x1 = total_units * (blockIdx.x + 1) / gridDim.x;
+    const bool word_ok = (reinterpret_cast<uintptr_t>(v_mask) & 3u) == 0 && (T & 1) == 0;
+    const int floor_k = min_per_token ? 1 : 0;
+    // nothing beyond the reserved groups is ever taken: no threshold, scan B alone
+    const bool select = k_nominal > floor_k;
+
+    // ---- scan A: histogram of the top 13 key bits of the sample's candidates ---------------------
+    const int per_unit = kUnit / samp;               // sampled tokens per unit
+    const int du = tid / per_unit, sidx = tid - du * per_unit;
+#pragma unroll 1
+    for (long long x = (skip_scan_a || !select) ? x1 : x0; x < x1;) {
+        const int problem = (int)(x / upp);
+        const int u0 = (int)(x - (long long)problem * upp);
+        const int n = (int)min((long long)(upp - u0), x1 - x);
+        x += n;
+        const int b = problem / Hkv, hk = problem - b * Hkv;
+        const int len = clamp_len(seq_len, b, T);
+        uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+        uint32_t* hist = hist_all + (size_t)problem * kBins13;
+        const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+        const float* rows = scores + (size_t)problem * T * S;
+        for (int i = tid; i < kBins13; i += kThreads) shist[i] = 0;
+        __syncthreads();
+        const uint32_t shist_base = smem_u32(shist);
+        uint32_t n_routed = 0;
+#pragma unroll 1
+        for (int v = u0; v < u0 + n; v += samp * kBatch) {
+            if (v * kUnit >= len) break;
+            uint4 raw[kBatch][S / 4];
+            bool routed[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {           // all of the thread's loads are in flight before the first use
+                // the thread's token of unit `unit`: run (sidx / 4) of the unit's sampled runs of four tokens;
+                // the runs of a unit start every 4 * samp tokens, shifted by the unit's number
+                const int unit = v + i * samp + du;
+                const int t = unit * kUnit + ((((sidx >> 2) * samp + (unit & (samp - 1))) << 2) | (sidx & 3));
+                routed[i] = unit < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
+                load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                n_routed += routed[i];
+                if (routed[i]) {
+                    uint32_t key[S];
+                    make_keys<S>(raw[i], key);
+#pragma unroll
+                    for (int j = 0; j < S; ++j) red_if(true, shist_base, key[j] >> kShift13, 1);
+                    red_if(min_per_token != 0, shist_base, max_key<S>(key) >> kShift13, -1);
+                }
+            }
+        }
+        __syncthreads();
+        for (int i = tid; i < kBins13; i += kThreads) {
+            const uint32_t v = shist[i];
+            if (v) atomicAdd(hist + i, v);
+        }
+        uint32_t tot;
+        block_excl_scan(n_routed, s_w, &tot);
+        if (tid == 0 && tot) atomicAdd(state + ST_NROUTEDA, tot);
+        __threadfence();
+        __syncthreads();
+        if (tid == 0)
+            s_last = (atomicAdd(state + ST_TICKETA, (unsigned)n) + (unsigned)n == (unsigned)upp);
+        __syncthreads();
+        if (!s_last) continue;
+        __threadfence();
+
+        // the CTA that completed the problem's sample derives the band and publishes it
+        const uint32_t n_s = __ldcg(state + ST_NROUTEDA);
+        const uint32_t m_c = n_s * (uint32_t)(S - floor_k);           // candidates in the sample
+        uint32_t b_lo = 0, b_hi = kBins13 - 1;
+        if (m_c > 0) {
+            float r_hi, r_lo;                                         // sample ranks (1 = largest) that bracket the threshold
+            if (samp == 1) {
+                r_hi = r_lo = (float)(n_s * (uint32_t)(k_nominal - floor_k));
+            } else {
+                const float f = (float)(k_nominal - floor_k) / (float)(S - floor_k);
+                const float r = f * (float)m_c;
+                const float d = 0.1f * (float)z_tenths * sqrtf((float)m_c * f * (1.f - f)) + 2.f;
+                r_hi = floorf(r - d);
+                r_lo = ceilf(r + d);
+            }
+            if (r_hi >= 1.f) {
+                pick_digit_n<false>(hist, kBins13, kBins13 / kThreads, (uint32_t)r_hi, s_w, s_pick);
+                b_hi = s_pick[0];
+                __syncthreads();
+            }
+            if (r_lo <= (float)m_c) {
+                pick_digit_n<false>(hist, kBins13, kBins13 / kThreads, (uint32_t)r_lo, s_w, s_pick);
+                b_lo = s_pick[0];
+                __syncthreads();
+            }
+        }
+        if (tid == 0) {
+            state[ST_BLO] = b_lo;
+            state[ST_BHI] = b_hi;
+            state[ST_PATH] = PATH_BAND;
+            __threadfence();
+            st_release(state + ST_DONEA, 1u);
+        }
+    }
+
+    // ---- scan B: definite bits above the band, the list inside it, counts ----------------------
+    constexpr int kTodoMax = 4;
+    __shared__ int s_todo[kTodoMax];                     // problems this CTA completed
+    int n_todo = 0;                                      // (the same in every thread)
+    auto settle = [&](int slot) {
+        __syncthreads();
+        const int problem = s_todo[slot];
+        __threadfence();
+        uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+        uint32_t flags = 0;
+        const uint32_t take = budget_of(__ldcg(state + ST_NROUTEDB), k_nominal, min_per_token, flags);
+        const uint32_t above = __ldcg(state + ST_ABOVE), listn = __ldcg(state + ST_LISTN);
+        if (flags || !select) {                          // nothing beyond the reserved groups (budget errors do not come here)
+            if (tid == 0) { state[ST_FLAGS] = flags; state[ST_KREM] = 0u; state[ST_PREFIX] = 0u; }
+        } else if (listn <= list_cap && above < take && take - above <= listn) {
+            if (tid == 0) state[ST_FLAGS] = 0u;
+            settle_band<S>(list_all + (size_t)problem * list_cap, listn, take - above, state,
+                           v_mask + (size_t)problem * T, tie_all + (size_t)problem * T,
+                           unit_sums + (size_t)problem * upp, word_ok, shist, s_w, s_pick);
+        } else if (tid == 0) {                           // the band missed the threshold, or the list overflowed
+            state[ST_PATH] = PATH_WIDE;
+            atomicExch(abort_word + 1, 1u);
+        }
+        __syncthreads();
+    };
+#pragma unroll 1
+    for (long long x = x0; x < x1;) {
+        const int problem = (int)(x / upp);
+        const int u0 = (int)(x - (long long)problem * upp);
+        const int n = (int)min((long long)(upp - u0), x1 - x);
+        x += n;
+        const int b = problem / Hkv, hk = problem - b * Hkv;
+        const int len = clamp_len(seq_len, b, T);
+        uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+        const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
+        uint4 raw[kBatch][S / 4];
+        int cls_of[kBatch];
+        const float* rows = scores + (size_t)problem * T * S;
+        uint2* list = list_all + (size_t)problem * list_cap;
+        auto load_batch = [&](int u) {
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int t = (u + i) * kUnit + tid;
+                cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
+                load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);
+            }
+        };
+        load_batch(u0);                                  // in flight while the band arrives
+        float lo = 0.f, hi = 0.f;
+        if (select) {
+            if (!wait_band(state, s_bc, abort_word, wait_ns)) return;
+            if (s_bc[1] != PATH_BAND) continue;
+            band_bounds(s_bc[2], s_bc[3], lo, hi);
+        }
+        uint32_t pend_n = 0, pend_base = 0;              // staged entries of the warp and (lane 31) their place in the list
+        auto flush = [&]() {
+            if (pend_n) {
+                __syncwarp();
+                const uint32_t base = __shfl_sync(0xFFFFFFFFu, pend_base, 31);
+                for (uint32_t e = lane; e < pend_n; e += 32)
+                    if (base + e < list_cap) list[base + e] = stage[e];
+                __syncwarp();
+                pend_n = 0;
+            }
+        };
+        if (tid < 2) s_cnt[tid] = 0u;                    // (ordered before the additions below by the barrier in wait_band
+        __syncthreads();                                 //  or this one)
+        uint32_t n_routed = 0, n_above = 0;
+#pragma unroll 1
+        for (int u = u0; u < u0 + n; u += kBatch) {
+            // 1. everything that needs the batch's scores: masks, counts, the list entries (to the staging slots)
+            uint32_t defs[kBatch], cands[kBatch], c_mine = 0;
+            bool in_range[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const int cl = cls_of[i];
+                defs[i] = 0;
+                cands[i] = 0;
+                if (cl == STC_CLS_FULL) {
+                    defs[i] = (1u << S) - 1u;
+                } else if (cl == STC_CLS_ROUTED) {
+                    band_token<S>(raw[i], select, lo, hi, min_per_token, defs[i], cands[i]);
+                    ++n_routed;
+                    n_above += __popc(defs[i]) - floor_k;
+                }
+                c_mine += __popc(cands[i]);
+                in_range[i] = u + i < u0 + n && (u + i) * kUnit + tid < T;
+            }
+            // The warp's candidates go to the list in one piece.  Its place there comes from an atomic addition
+            // whose answer takes a microsecond: the entries wait in the warp's staging slots and are written out
+            // one batch later, when the answer has long arrived.
+            flush();
+            const uint32_t incl = warp_incl_scan(c_mine, lane);
+            const uint32_t w_total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            const bool staged = w_total <= (uint32_t)kStage;
+            if (w_total) {
+                uint32_t pos = incl - c_mine;
+                if (!staged) {                           // (too many for the slots: rare; wait for the place)
+                    uint32_t base = 0;
+                    if (lane == 31) base = atomicAdd(state + ST_LISTN, w_total);
+                    pos += __shfl_sync(0xFFFFFFFFu, base, 31);
+                }
+                uint2* dst = staged ? stage : list;
+                const uint32_t lim = staged ? (uint32_t)kStage : list_cap;
+#pragma unroll
+                for (int i = 0; i < kBatch; ++i) {
+                    uint32_t m = cands[i];
+                    const uint32_t flat = (uint32_t)((u + i) * kUnit + tid) * S;
+                    while (m) {
+                        const int j = __ffs(m) - 1;
+                        m &= m - 1;
+                        if (pos < lim)
+                            dst[pos] = make_uint2(float_key(__uint_as_float(raw_word<S>(raw[i], j))), flat + j);
+                        ++pos;
+                    }
+                }
+            }
+            // 2. the scores are no longer needed: the next batch's loads go out now and fly during the rest
+            if (u + kBatch < u0 + n) load_batch(u + kBatch);
+            // 3. what only needs the masks
+            if (w_total && staged) {
+                if (lane == 31) pend_base = atomicAdd(state + ST_LISTN, w_total);
+                pend_n = w_total;
+            }
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                if (in_range[i]) {
+                    const size_t at = (size_t)problem * T + (size_t)(u + i) * kUnit + tid;
+                    v_mask[at] = (uint16_t)defs[i];
+                    tie_all[at] = 0;
+                }
+                // per-unit count of definite bits: the unit's word starts at zero (the call's clear) and only
+                // ever receives additions, from here and from the CTA that settles the list
+                const uint32_t cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(defs[i]));
+                if (lane == 0 && cnt && u + i < u0 + n) atomicAdd(unit_sums + (size_t)problem * upp + u + i, cnt);
+            }
+        }
+        flush();
+        n_routed = __reduce_add_sync(0xFFFFFFFFu, n_routed);
+        n_above = __reduce_add_sync(0xFFFFFFFFu, n_above);
+        if (lane == 0) { atomicAdd(&s_cnt[0], n_routed); atomicAdd(&s_cnt[1], n_above); }
+        __syncthreads();
+        if (tid == 0) {
+            if (s_cnt[0]) atomicAdd(state + ST_NROUTEDB, s_cnt[0]);
+            if (s_cnt[1]) atomicAdd(state + ST_ABOVE, s_cnt[1]);
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0)
+            s_last = (atomicAdd(state + ST_TICKETB, (unsigned)n) + (unsigned)n == (unsigned)upp);
+        __syncthreads();
+        if (!s_last) continue;
+        // this CTA completed scan B of the problem and settles it -- once its own scanning is over, so that the
+        // problems it still has units of are not held up (a full to-do list is worked off at once)
+        if (tid == 0) s_todo[n_todo] = problem;
+        if (++n_todo == kTodoMax) {
+            for (int i = 0; i < n_todo; ++i) settle(i);
+            n_todo = 0;
+        }
+    }
+    for (int i = 0; i < n_todo; ++i) settle(i);
 }
 
 // Problems of at most kBatch units (one token per thread and unit): a CTA takes whole
@@ -724,13 +1270,11 @@ size_t route_ws_bytes(const Geom& g) { return carve(g, nullptr).total_bytes; }
 
 namespace {
 
-// CTAs of the select kernel that can be resident at once (it is launched cooperatively).
-template <int S>
-cudaError_t select_grid_limit(int* limit) {
-    // per device: the occupancy of the kernel is a property of the kernel and the device, the
+// CTAs of a cooperatively launched kernel that can be resident at once.
+cudaError_t coop_grid_limit(const void* fn, std::atomic<int>* cached /*[kMaxDevices]*/, int* limit) {
+    // per device: the occupancy of a kernel is a property of the kernel and the device, the
     // query is cheap next to a cooperative launch, and a process may drive several devices
     constexpr int kMaxDevices = 64;
-    static std::atomic<int> cached[kMaxDevices];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
@@ -738,8 +1282,7 @@ cudaError_t select_grid_limit(int* limit) {
     if (v == 0) {
         int sms = 0, per_sm = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess)
-            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, route_select_kernel<S>, kThreads, 0);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, 0);
         if (e != cudaSuccess) return e;
         if (sms <= 0 || per_sm <= 0) return cudaErrorLaunchOutOfResources;
         v = sms * per_sm;
@@ -753,20 +1296,56 @@ template <int S>
 cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls, int64_t cls_b, int64_t cls_h,
                           int k_nominal, int min_per_token, int mode, const RouteWs& w, uint16_t* v_mask,
                           cudaStream_t st) {
-    int limit = 0;
-    cudaError_t e = select_grid_limit<S>(&limit);
-    if (e != cudaSuccess) return e;
+    static std::atomic<int> cached_select[64], cached_band[64];
     int upp = (g.T + kUnit - 1) / kUnit;
     long long total_units = (long long)upp * g.problems;
-    const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
     const int32_t* seq_len = g.seq_len;
     int Hkv = g.Hkv, T = g.T;
-    uint32_t *state = w.state, *hist = w.hist, *abort_word = w.abort_word, *unit_sums = w.unit_sums;
+    uint32_t *state = w.state, *hist = w.hist, *hist13 = w.hist13, *abort_word = w.abort_word, *unit_sums = w.unit_sums;
     uint16_t* tie = w.tie;
-    int first_pass = g_first_pass.load();
+    uint2* list = w.list;
+    uint32_t list_cap = w.list_cap;
+    const int knob = g_first_pass.load();
     unsigned long long wait_ns = g_wait_ns.load();
+    // The band kernel settles the global budget in two scans; the multi-pass kernel follows for the problems
+    // it left (it returns at once when there is none) and does everything in PER_TOKEN mode.
+    // (a floor of one group per token with a nominal budget of none is the budget error: the multi-pass kernel reports it)
+    // It pays when the scores do not stay in L2 between the scans (each of the four passes of the multi-pass
+    // kernel is then a trip to HBM); smaller score arrays are quicker with the multi-pass kernel.
+    bool big = false;
+    {
+        int dev = 0, l2 = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) == cudaSuccess)
+            big = (double)g.problems * g.T * g.S * 4.0 >= 2.0 * (double)l2;
+    }
+    const bool band = mode == STC_MODE_GLOBAL && ((knob == 0 && big) || knob >= 4) &&
+                      !(min_per_token && k_nominal == 0);
+    cudaError_t e;
+    int limit = 0;
+    if (band) {
+        e = coop_grid_limit(reinterpret_cast<const void*>(route_band_kernel<S>), cached_band, &limit);
+        if (e != cudaSuccess) return e;
+        const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
+        int skip_scan_a = knob == 4;
+        // scan A samples one token in `samp`, keeping at least 2^17 keys of a problem in the sample
+        const long long keys = (long long)g.T * g.S;
+        int samp = knob == 5 ? 1 : (keys >= (1 << 20) ? 8 : keys >= (1 << 19) ? 4 : keys >= (1 << 18) ? 2 : 1);
+        int z_tenths = knob == 6 ? 0 : 50;
+        void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token,
+                        &state, &hist13, &abort_word, &v_mask, &tie, &unit_sums, &list, &list_cap, &total_units,
+                        &skip_scan_a, &wait_ns, &samp, &z_tenths};
+        e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_band_kernel<S>), dim3(grid), dim3(kThreads),
+                                        args, 0, st);
+        if (e != cudaSuccess) return e;
+    }
+    e = coop_grid_limit(reinterpret_cast<const void*>(route_select_kernel<S>), cached_select, &limit);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
+    int first_pass = (knob >= 1 && knob <= 3) ? knob : 0;
+    int only_wide = band;
     void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token, &mode,
-                    &state, &hist, &abort_word, &v_mask, &tie, &unit_sums, &total_units, &first_pass, &wait_ns};
+                    &state, &hist, &abort_word, &v_mask, &tie, &unit_sums, &total_units, &first_pass, &wait_ns,
+                    &only_wide};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_select_kernel<S>), dim3(grid),
                                        dim3(kThreads), args, 0, st);
 }
@@ -822,17 +1401,23 @@ cudaError_t launch_route_pack(const Geom& g, const void* v, const float* scores,
 }
 
 void set_route_select_knobs(int first_pass, unsigned long long wait_ns) {
-    g_first_pass.store(first_pass < 0 || first_pass > 3 ? 0 : first_pass);
+    g_first_pass.store(first_pass < -1 || first_pass > 7 ? 0 : first_pass);
     g_wait_ns.store(wait_ns ? wait_ns : kWaitNs);
 }
 
 }  // namespace stc
 
-// Test hook, not part of the public interface (not declared in stc.h): makes the cooperative
-// selection kernel start at histogram pass `first_pass` (0 = normal) and bound its hand-off waits by
-// wait_ns (0 = the default of two seconds).  With first_pass = 3 on a freshly cleared workspace no
-// CTA ever publishes a digit, so every wait runs into its limit and the give-up path (abort word,
-// orderly return, STC_ERR_TIMEOUT from the packing kernel) executes without anything hanging.
+// Test hook, not part of the public interface (not declared in stc.h).  first_pass: 0 = normal (for score
+// arrays well beyond the L2 size the band kernel, then the multi-pass kernel for what it left; else the
+// multi-pass kernel alone); -1 = the multi-pass kernel alone; 1..3 = the
+// multi-pass kernel alone, starting at that histogram pass; 4 = the band kernel without its first scan;
+// 5 = the band kernel with every token in its sample (the band is then exact); 6 = the band kernel with
+// a band of almost no width (it misses often, and the multi-pass kernel then redoes those problems);
+// 7 = the band kernel as in production, whatever the size of the call.
+// wait_ns bounds the hand-off waits (0 = the default of two seconds).  With first_pass = 3 or 4 on a
+// freshly cleared workspace no CTA ever publishes a digit, so every wait runs into its limit and the
+// give-up path (abort word, orderly return, STC_ERR_TIMEOUT from the packing kernel) executes without
+// anything hanging.
 extern "C" void stc_test_route_select_knobs(int32_t first_pass, uint64_t wait_ns) {
     stc::set_route_select_knobs(first_pass, wait_ns);
 }
