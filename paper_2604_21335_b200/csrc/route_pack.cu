@@ -55,7 +55,7 @@ struct RouteWs {
     uint32_t* hist;       // [problems][3][kBins]
     uint32_t* hist13;     // [problems][kBins13]
     uint32_t* abort_word; // set when a bounded wait gave up; the next word: some problem is left to the multi-pass kernel
-    uint2* list;          // [problems][list_cap] (key, flat index) of the candidates in the threshold's bin
+    uint2* list;          // [problems][list_cap] (score bits, flat index) of the candidates inside the band
     uint32_t list_cap;
     uint32_t* unit_sums;  // [problems][units]: definite count | tie count << 16 (the band kernel adds to zeroed words)
     uint16_t* tie;        // [problems][T]
@@ -540,12 +540,12 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
 //   written straight away and counted), those below are dropped, those inside -- a per cent or two
 //   of the problem -- are appended as (key, flat index) pairs to the problem's list.  All tests are
 //   float comparisons against the band's two edges; keys are only built for the list.
-//   The CTA that completes scan B of a problem settles it exactly: with `above` pairs counted above
-//   the band, the take-th largest candidate is the (take - above)-th largest of the list, provided
-//   above < take <= above + list length -- which is the check that the band was right.  Radix select
-//   over the list (three passes, the list sits in L2), then one pass that sets the definite bit of
-//   every listed pair above the threshold and the tie bit of every pair on it (the compaction
-//   resolves ties in flat-index order, as after the multi-pass kernel).
+//   The settle kernel (next launch, one CTA per problem) settles each problem exactly: with `above`
+//   pairs counted above the band, the take-th largest candidate is the (take - above)-th largest of
+//   the list, provided above < take <= above + list length -- which is the check that the band was
+//   right.  Radix select over the list, then one pass that sets the definite bit of every listed pair
+//   above the threshold and the tie bit of every pair on it (the compaction resolves ties in
+//   flat-index order, as after the multi-pass kernel).
 // A problem whose band was wrong, or holds more pairs than the list has room for (massive ties), is
 // marked PATH_WIDE and left to the multi-pass kernel that runs next; the result is the same either way.
 
@@ -698,63 +698,128 @@ __device__ __forceinline__ void band_token(const uint4 (&raw)[S / 4], bool selec
     }
 }
 
-// Key j of a token's raw scores (j known at run time: selected by value, no indexed registers).
-template <int S>
-__device__ __forceinline__ uint32_t raw_word(const uint4 (&raw)[S / 4], int j) {
-    uint32_t w = 0;
-#pragma unroll
-    for (int i = 0; i < S / 4; ++i) {
-        w = j == 4 * i + 0 ? raw[i].x : w;
-        w = j == 4 * i + 1 ? raw[i].y : w;
-        w = j == 4 * i + 2 ? raw[i].z : w;
-        w = j == 4 * i + 3 ? raw[i].w : w;
+// ---- the settle kernel: one CTA of 1024 threads per problem, after the band kernel -------------
+// Checks the band (above < take <= above + list length), finds the (take - above)-th largest key of the
+// list by radix select (11 + 11 + 10 bits; the keys are staged in shared memory when they fit, else every
+// pass reads the list, which sits in L2), then sets the definite bit of every listed pair above the
+// threshold and the tie bit of every pair on it, and adds them to the per-unit counts.
+constexpr int kSettleThreads = 1024;
+constexpr int kSettleWarps = kSettleThreads / 32;
+constexpr int kSettleKeys = 45056;                 // keys staged in shared memory (176 KiB)
+constexpr size_t kSettleSmem = (size_t)kSettleKeys * 4;
+
+// Exclusive scan of one value per thread over the settle kernel's CTA.
+__device__ __forceinline__ uint32_t settle_excl_scan(uint32_t v, uint32_t* s_w /*[kSettleWarps]*/) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t incl = warp_incl_scan(v, lane);
+    __syncthreads();
+    if (lane == 31) s_w[warp] = incl;
+    __syncthreads();
+    uint32_t base = 0;
+    for (int w = 0; w < warp; ++w) base += s_w[w];
+    return base + incl - v;
+}
+// The bin holding the krem-th largest count of a shared-memory histogram (thread t owns the `per` bins
+// nbins-1-per*t downwards; nbins = per * kSettleThreads).  s_out = {bin, rank inside it}.
+__device__ __forceinline__ void settle_pick(const uint32_t* hist, int nbins, int per, uint32_t krem, uint32_t* s_w,
+                                            uint32_t* s_out) {
+    const int top = nbins - 1 - per * (int)threadIdx.x;
+    uint32_t sum = 0;
+    for (int j = 0; j < per; ++j) sum += hist[top - j];
+    const uint32_t excl = settle_excl_scan(sum, s_w);
+    if (excl < krem && krem <= excl + sum) {
+        uint32_t run = excl;
+        for (int j = 0; j < per; ++j) {
+            const uint32_t c = hist[top - j];
+            if (run + c >= krem) { s_out[0] = (uint32_t)(top - j); s_out[1] = krem - run; break; }
+            run += c;
+        }
     }
-    return w;
+    __syncthreads();
 }
 
-// The list of a problem is complete: find the krem-th largest of its keys and set the bits.
 template <int S>
-__device__ __noinline__ void settle_band(const uint2* __restrict__ list, uint32_t n_list, uint32_t krem,
-                                         uint32_t* __restrict__ state, uint16_t* __restrict__ mask_row,
-                                         uint16_t* __restrict__ tie_row, uint32_t* __restrict__ sums_row,
-                                         bool word_ok, uint32_t* shist, uint32_t* s_w, uint32_t* s_pick) {
+__global__ void __launch_bounds__(kSettleThreads, 1)
+route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abort_word,
+                    const uint2* __restrict__ list_all, uint32_t list_cap, uint16_t* __restrict__ v_mask,
+                    uint16_t* __restrict__ tie_all, uint32_t* __restrict__ unit_sums, int T, int upp,
+                    int k_nominal, int min_per_token) {
+    extern __shared__ __align__(16) uint32_t s_keys[];
+    __shared__ uint32_t shist[2048];
+    __shared__ uint32_t s_w[kSettleWarps];
+    __shared__ uint32_t s_pick[2];
     const int tid = threadIdx.x;
-    constexpr int kInFlight = 16;                   // list entries a thread has in flight (the list sits in L2)
-    uint32_t prefix = 0;
+    const int problem = blockIdx.x;
+    uint32_t* state = state_all + (size_t)problem * ST_WORDS;
+    if (__ldcg(abort_word) != 0u || __ldcg(state + ST_PATH) != PATH_BAND) return;   // a wait gave up: nothing is settled
+    const bool select = k_nominal > (min_per_token ? 1 : 0);
+    uint32_t flags = 0;
+    const uint32_t take = budget_of(__ldcg(state + ST_NROUTEDB), k_nominal, min_per_token, flags);
+    const uint32_t above = __ldcg(state + ST_ABOVE), n_list = __ldcg(state + ST_LISTN);
+    if (flags || !select) {                              // nothing beyond the reserved groups (budget errors do not come here)
+        if (tid == 0) { state[ST_FLAGS] = flags; state[ST_KREM] = 0u; state[ST_PREFIX] = 0u; }
+        return;
+    }
+    if (!(n_list <= list_cap && above < take && take - above <= n_list)) {
+        if (tid == 0) {                                  // the band missed the threshold, or the list overflowed
+            state[ST_PATH] = PATH_WIDE;
+            atomicExch(abort_word + 1, 1u);
+        }
+        return;
+    }
+    const uint2* list = list_all + (size_t)problem * list_cap;
+    const bool word_ok = (reinterpret_cast<uintptr_t>(v_mask) & 3u) == 0 && (T & 1) == 0;
+    uint16_t* mask_row = v_mask + (size_t)problem * T;
+    uint16_t* tie_row = tie_all + (size_t)problem * T;
+    uint32_t* sums_row = unit_sums + (size_t)problem * upp;
+    constexpr int kInFlight = 8;                         // list entries a thread has in flight
+    const bool staged = n_list <= (uint32_t)kSettleKeys;
+    if (staged) {
 #pragma unroll 1
-    for (int pass = 0; pass < 3; ++pass) {          // 11 + 11 + 10 bits
+        for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kSettleThreads) {
+            uint32_t w[kInFlight];
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i) w[i] = __ldcg(&list[min(e0 + i * kSettleThreads, n_list - 1)].x);
+#pragma unroll
+            for (int i = 0; i < kInFlight; ++i)
+                if (e0 + i * kSettleThreads < n_list) s_keys[e0 + i * kSettleThreads] = float_key(__uint_as_float(w[i]));
+        }
+    }
+    auto key_at = [&](uint32_t e) {
+        return staged ? s_keys[e] : float_key(__uint_as_float(__ldcg(&list[e].x)));
+    };
+    uint32_t prefix = 0, krem = take - above;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {               // 11 + 11 + 10 bits
         const uint32_t himask = pass_himask(pass);
         const int dshift = pass_shift(pass);
         const int nbins = pass == 2 ? 1024 : 2048;
-        for (int i = tid; i < nbins; i += kThreads) shist[i] = 0u;
+        for (int i = tid; i < nbins; i += kSettleThreads) shist[i] = 0u;
         __syncthreads();
-#pragma unroll 1
-        for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kThreads) {
-            uint32_t k[kInFlight];
-#pragma unroll
-            for (int i = 0; i < kInFlight; ++i) k[i] = __ldcg(&list[min(e0 + i * kThreads, n_list - 1)].x);
-#pragma unroll
-            for (int i = 0; i < kInFlight; ++i)
-                if (e0 + i * kThreads < n_list && (k[i] & himask) == prefix)
-                    atomicAdd(&shist[(k[i] >> dshift) & (uint32_t)(nbins - 1)], 1u);
+#pragma unroll 4
+        for (uint32_t e = tid; e < n_list; e += kSettleThreads) {
+            const uint32_t k = key_at(e);
+            if ((k & himask) == prefix) atomicAdd(&shist[(k >> dshift) & (uint32_t)(nbins - 1)], 1u);
         }
         __syncthreads();
-        pick_digit_n<true>(shist, nbins, nbins / kThreads, krem, s_w, s_pick);
+        settle_pick(shist, nbins, nbins / kSettleThreads, krem, s_w, s_pick);
         prefix |= s_pick[0] << dshift;
         krem = s_pick[1];
         __syncthreads();
     }
-    const uint32_t tau = prefix;                    // krem: how many of the pairs on the threshold are kept
+    const uint32_t tau = prefix;                         // krem: how many of the pairs on the threshold are kept
 #pragma unroll 1
-    for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kThreads) {
+    for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kSettleThreads) {
         uint2 en[kInFlight];
 #pragma unroll
-        for (int i = 0; i < kInFlight; ++i) en[i] = __ldcg(&list[min(e0 + i * kThreads, n_list - 1)]);
+        for (int i = 0; i < kInFlight; ++i) en[i] = __ldcg(&list[min(e0 + i * kSettleThreads, n_list - 1)]);
 #pragma unroll
         for (int i = 0; i < kInFlight; ++i) {
-            if (e0 + i * kThreads >= n_list || en[i].x < tau) continue;
+            const uint32_t key = float_key(__uint_as_float(en[i].x));
+            if (e0 + i * kSettleThreads >= n_list || key < tau) continue;
             const uint32_t t = en[i].y / S, j = en[i].y - t * S;
-            if (en[i].x > tau) {
+            if (t >= (uint32_t)T) continue;              // (cannot happen: the scan wrote the entry)
+            if (key > tau) {
                 or16(mask_row + t, 1u << j, word_ok);
                 atomicAdd(sums_row + t / kUnit, 1u);
             } else {
@@ -763,7 +828,7 @@ __device__ __noinline__ void settle_band(const uint2* __restrict__ list, uint32_
             }
         }
     }
-    if (tid == 0) { state[ST_PREFIX] = tau; state[ST_KREM] = krem; }
+    if (tid == 0) { state[ST_FLAGS] = 0u; state[ST_PREFIX] = tau; state[ST_KREM] = krem; }
 }
 
 // samp: 1, 2, 4 or 8 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
@@ -778,7 +843,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                   uint32_t* __restrict__ unit_sums, uint2* __restrict__ list_all, uint32_t list_cap,
                   long long total_units, int skip_scan_a, unsigned long long wait_ns, int samp, int z_tenths) {
     constexpr int kBatch = S >= 8 ? 32 / S : 4;  // tokens in flight per thread (at most 32 score registers)
-    __shared__ uint32_t shist[kBins13];
+    __shared__ __align__(16) uint32_t shist[kBins13];
     __shared__ uint32_t s_w[kWarps];
     __shared__ uint32_t s_pick[3];
     __shared__ uint32_t s_bc[4];
@@ -786,12 +851,16 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
     __shared__ int s_last;
     constexpr int kStage = 64;                   // list entries a warp can hold back
     __shared__ uint2 s_stage[kWarps][kStage];
+    // scan B has no use for the histogram: its words hold the segment's per-unit counts and one scratch row per thread
+    constexpr int kUnitsMax = 2048;
+    static_assert(kUnitsMax + kThreads * S <= kBins13, "scan B's scratch fits the histogram");
+    uint32_t* s_units = shist;
+    uint32_t* s_row = shist + kUnitsMax + threadIdx.x * S;
 
     const int tid = threadIdx.x, lane = tid & 31;
     uint2* stage = s_stage[tid >> 5];
     const long long x0 = total_units * blockIdx.x / gridDim.x;
     const long long x1 = total_units * (blockIdx.x + 1) / gridDim.x;
-    const bool word_ok = (reinterpret_cast<uintptr_t>(v_mask) & 3u) == 0 && (T & 1) == 0;
     const int floor_k = min_per_token ? 1 : 0;
     // nothing beyond the reserved groups is ever taken: no threshold, scan B alone
     const bool select = k_nominal > floor_k;
@@ -893,35 +962,11 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
     }
 
     // ---- scan B: definite bits above the band, the list inside it, counts ----------------------
-    constexpr int kTodoMax = 4;
-    __shared__ int s_todo[kTodoMax];                     // problems this CTA completed
-    int n_todo = 0;                                      // (the same in every thread)
-    auto settle = [&](int slot) {
-        __syncthreads();
-        const int problem = s_todo[slot];
-        __threadfence();
-        uint32_t* state = state_all + (size_t)problem * ST_WORDS;
-        uint32_t flags = 0;
-        const uint32_t take = budget_of(__ldcg(state + ST_NROUTEDB), k_nominal, min_per_token, flags);
-        const uint32_t above = __ldcg(state + ST_ABOVE), listn = __ldcg(state + ST_LISTN);
-        if (flags || !select) {                          // nothing beyond the reserved groups (budget errors do not come here)
-            if (tid == 0) { state[ST_FLAGS] = flags; state[ST_KREM] = 0u; state[ST_PREFIX] = 0u; }
-        } else if (listn <= list_cap && above < take && take - above <= listn) {
-            if (tid == 0) state[ST_FLAGS] = 0u;
-            settle_band<S>(list_all + (size_t)problem * list_cap, listn, take - above, state,
-                           v_mask + (size_t)problem * T, tie_all + (size_t)problem * T,
-                           unit_sums + (size_t)problem * upp, word_ok, shist, s_w, s_pick);
-        } else if (tid == 0) {                           // the band missed the threshold, or the list overflowed
-            state[ST_PATH] = PATH_WIDE;
-            atomicExch(abort_word + 1, 1u);
-        }
-        __syncthreads();
-    };
 #pragma unroll 1
     for (long long x = x0; x < x1;) {
         const int problem = (int)(x / upp);
         const int u0 = (int)(x - (long long)problem * upp);
-        const int n = (int)min((long long)(upp - u0), x1 - x);
+        const int n = (int)min((long long)min(upp - u0, kUnitsMax), x1 - x);   // (its unit counts fit the scratch)
         x += n;
         const int b = problem / Hkv, hk = problem - b * Hkv;
         const int len = clamp_len(seq_len, b, T);
@@ -957,14 +1002,14 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                 pend_n = 0;
             }
         };
-        if (tid < 2) s_cnt[tid] = 0u;                    // (ordered before the additions below by the barrier in wait_band
-        __syncthreads();                                 //  or this one)
+        if (tid < 2) s_cnt[tid] = 0u;
+        for (int i = tid; i < n; i += kThreads) s_units[i] = 0u;
+        __syncthreads();
         uint32_t n_routed = 0, n_above = 0;
 #pragma unroll 1
         for (int u = u0; u < u0 + n; u += kBatch) {
             // 1. everything that needs the batch's scores: masks, counts, the list entries (to the staging slots)
             uint32_t defs[kBatch], cands[kBatch], c_mine = 0;
-            bool in_range[kBatch];
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
                 const int cl = cls_of[i];
@@ -978,7 +1023,6 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                     n_above += __popc(defs[i]) - floor_k;
                 }
                 c_mine += __popc(cands[i]);
-                in_range[i] = u + i < u0 + n && (u + i) * kUnit + tid < T;
             }
             // The warp's candidates go to the list in one piece.  Its place there comes from an atomic addition
             // whose answer takes a microsecond: the entries wait in the warp's staging slots and are written out
@@ -999,12 +1043,15 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) {
                     uint32_t m = cands[i];
+                    if (m == 0u) continue;               // (nine tokens in ten)
+                    // the token's scores go to the thread's scratch row, where a score can be picked by number
+#pragma unroll
+                    for (int q = 0; q < S / 4; ++q) reinterpret_cast<uint4*>(s_row)[q] = raw[i][q];
                     const uint32_t flat = (uint32_t)((u + i) * kUnit + tid) * S;
                     while (m) {
                         const int j = __ffs(m) - 1;
                         m &= m - 1;
-                        if (pos < lim)
-                            dst[pos] = make_uint2(float_key(__uint_as_float(raw_word<S>(raw[i], j))), flat + j);
+                        if (pos < lim) dst[pos] = make_uint2(s_row[j], flat + j);   // (score bits, flat index)
                         ++pos;
                     }
                 }
@@ -1018,15 +1065,14 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             }
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
-                if (in_range[i]) {
+                if (u + i < u0 + n && (u + i) * kUnit + tid < T) {
                     const size_t at = (size_t)problem * T + (size_t)(u + i) * kUnit + tid;
                     v_mask[at] = (uint16_t)defs[i];
                     tie_all[at] = 0;
                 }
-                // per-unit count of definite bits: the unit's word starts at zero (the call's clear) and only
-                // ever receives additions, from here and from the CTA that settles the list
+                // per-unit count of definite bits, gathered in shared memory for the whole segment
                 const uint32_t cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(defs[i]));
-                if (lane == 0 && cnt && u + i < u0 + n) atomicAdd(unit_sums + (size_t)problem * upp + u + i, cnt);
+                if (lane == 0 && cnt && u + i < u0 + n) atomicAdd(&s_units[u + i - u0], cnt);
             }
         }
         flush();
@@ -1038,21 +1084,10 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             if (s_cnt[0]) atomicAdd(state + ST_NROUTEDB, s_cnt[0]);
             if (s_cnt[1]) atomicAdd(state + ST_ABOVE, s_cnt[1]);
         }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0)
-            s_last = (atomicAdd(state + ST_TICKETB, (unsigned)n) + (unsigned)n == (unsigned)upp);
-        __syncthreads();
-        if (!s_last) continue;
-        // this CTA completed scan B of the problem and settles it -- once its own scanning is over, so that the
-        // problems it still has units of are not held up (a full to-do list is worked off at once)
-        if (tid == 0) s_todo[n_todo] = problem;
-        if (++n_todo == kTodoMax) {
-            for (int i = 0; i < n_todo; ++i) settle(i);
-            n_todo = 0;
-        }
+        // (plain stores: the settle kernel, which runs after this one, adds the listed pairs it keeps)
+        for (int i = tid; i < n; i += kThreads) unit_sums[(size_t)problem * upp + u0 + i] = s_units[i];
+        __syncthreads();                                 // the scratch is reused by the next segment
     }
-    for (int i = 0; i < n_todo; ++i) settle(i);
 }
 
 // Problems of at most kBatch units (one token per thread and unit): a CTA takes whole
@@ -1336,6 +1371,12 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
                         &skip_scan_a, &wait_ns, &samp, &z_tenths};
         e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_band_kernel<S>), dim3(grid), dim3(kThreads),
                                         args, 0, st);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(route_settle_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSettleSmem);
+        if (e != cudaSuccess) return e;
+        route_settle_kernel<S><<<(unsigned)g.problems, kSettleThreads, kSettleSmem, st>>>(
+            state, abort_word, list, list_cap, v_mask, tie, unit_sums, T, upp, k_nominal, min_per_token);
+        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     e = coop_grid_limit(reinterpret_cast<const void*>(route_select_kernel<S>), cached_select, &limit);
