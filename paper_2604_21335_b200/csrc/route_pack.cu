@@ -6,6 +6,11 @@
 // the lower flat index.  `take` depends on the routed-token count, which only
 // the device knows, so everything is resolved on the device:
 //
+//   GLOBAL budget, score arrays of at least twice the L2 size: the band kernel and the
+//   settle kernel (described where they are defined, further down) find the threshold in
+//   one scan of the scores plus a sampled one; the multi-pass kernel below then only
+//   redoes the problems they could not settle.  Otherwise:
+//
 //   select kernel (one persistent cooperative launch):
 //   hist pass 0/1/2  radix select (11+11+10 bits) of the take-th largest key
 //                    among the candidates; each CTA histograms its units of a
@@ -21,8 +26,9 @@
 //                    written, kept 16-byte chunks of V copied to the store.
 //
 // PER_TOKEN mode skips the histogram passes (the mask is local to a token).
-// HBM traffic: scores 4x (3 passes + mask, from L2 when they fit; 1x in PER_TOKEN
-// mode), kept part of V once in and once out.
+// HBM traffic: scores 4x in the multi-pass kernel (3 passes + mask, from L2 when they
+// fit), 1x plus the sample in the band kernel, 1x in PER_TOKEN mode; kept part of V once
+// in and once out.
 #include <atomic>
 
 #include "common.cuh"
@@ -708,7 +714,7 @@ constexpr int kSettleWarps = kSettleThreads / 32;
 constexpr int kSettleKeys = 45056;                 // keys staged in shared memory (176 KiB)
 constexpr size_t kSettleSmem = (size_t)kSettleKeys * 4;
 
-// Exclusive scan of one value per thread over the settle kernel's CTA.
+// Exclusive scan of one value per thread over a CTA of 1024 threads (the band and the settle kernel).
 __device__ __forceinline__ uint32_t settle_excl_scan(uint32_t v, uint32_t* s_w /*[kSettleWarps]*/) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t incl = warp_incl_scan(v, lane);
@@ -719,20 +725,33 @@ __device__ __forceinline__ uint32_t settle_excl_scan(uint32_t v, uint32_t* s_w /
     for (int w = 0; w < warp; ++w) base += s_w[w];
     return base + incl - v;
 }
-// The bin holding the krem-th largest count of a shared-memory histogram (thread t owns the `per` bins
-// nbins-1-per*t downwards; nbins = per * kSettleThreads).  s_out = {bin, rank inside it}.
+// The bin holding the krem-th largest count of a histogram (thread t owns the `per` bins nbins-1-per*t
+// downwards; nbins = per * 1024; kGlobal: the histogram is in global memory and per = 8, read as two
+// 16-byte pieces).  s_out = {bin, rank inside it}.
+template <bool kGlobal>
 __device__ __forceinline__ void settle_pick(const uint32_t* hist, int nbins, int per, uint32_t krem, uint32_t* s_w,
                                             uint32_t* s_out) {
     const int top = nbins - 1 - per * (int)threadIdx.x;
+    uint32_t c[8];
+    if (kGlobal) {
+        const uint4 a = __ldcg(reinterpret_cast<const uint4*>(hist + top - 7));
+        const uint4 b = __ldcg(reinterpret_cast<const uint4*>(hist + top - 3));
+        c[7] = a.x; c[6] = a.y; c[5] = a.z; c[4] = a.w; c[3] = b.x; c[2] = b.y; c[1] = b.z; c[0] = b.w;   // c[j] = bin top - j
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c[j] = j < per ? hist[top - j] : 0u;
+    }
     uint32_t sum = 0;
-    for (int j = 0; j < per; ++j) sum += hist[top - j];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum += c[j];
     const uint32_t excl = settle_excl_scan(sum, s_w);
     if (excl < krem && krem <= excl + sum) {
         uint32_t run = excl;
-        for (int j = 0; j < per; ++j) {
-            const uint32_t c = hist[top - j];
-            if (run + c >= krem) { s_out[0] = (uint32_t)(top - j); s_out[1] = krem - run; break; }
-            run += c;
+        bool found = false;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (!found && run + c[j] >= krem) { s_out[0] = (uint32_t)(top - j); s_out[1] = krem - run; found = true; }
+            run += c[j];
         }
     }
     __syncthreads();
@@ -802,12 +821,16 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
             if ((k & himask) == prefix) atomicAdd(&shist[(k >> dshift) & (uint32_t)(nbins - 1)], 1u);
         }
         __syncthreads();
-        settle_pick(shist, nbins, nbins / kSettleThreads, krem, s_w, s_pick);
+        settle_pick<false>(shist, nbins, nbins / kSettleThreads, krem, s_w, s_pick);
         prefix |= s_pick[0] << dshift;
         krem = s_pick[1];
         __syncthreads();
     }
     const uint32_t tau = prefix;                         // krem: how many of the pairs on the threshold are kept
+    // the per-unit counts of what is added are gathered in the histogram's words when the problem's units fit there
+    const bool local_sums = upp <= 2048;
+    if (local_sums) for (int i = tid; i < upp; i += kSettleThreads) shist[i] = 0u;
+    __syncthreads();
 #pragma unroll 1
     for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kSettleThreads) {
         uint2 en[kInFlight];
@@ -819,13 +842,17 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
             if (e0 + i * kSettleThreads >= n_list || key < tau) continue;
             const uint32_t t = en[i].y / S, j = en[i].y - t * S;
             if (t >= (uint32_t)T) continue;              // (cannot happen: the scan wrote the entry)
-            if (key > tau) {
-                or16(mask_row + t, 1u << j, word_ok);
-                atomicAdd(sums_row + t / kUnit, 1u);
-            } else {
-                or16(tie_row + t, 1u << j, word_ok);
-                atomicAdd(sums_row + t / kUnit, 1u << 16);
-            }
+            const uint32_t add = key > tau ? 1u : 1u << 16;
+            or16((key > tau ? mask_row : tie_row) + t, 1u << j, word_ok);
+            if (local_sums) atomicAdd(&shist[t / kUnit], add);
+            else atomicAdd(sums_row + t / kUnit, add);
+        }
+    }
+    if (local_sums) {
+        __syncthreads();
+        for (int i = tid; i < upp; i += kSettleThreads) {       // (nobody else touches the problem's counts now)
+            const uint32_t v = shist[i];
+            if (v) sums_row[i] += v;
         }
     }
     if (tid == 0) { state[ST_FLAGS] = 0u; state[ST_PREFIX] = tau; state[ST_KREM] = krem; }
@@ -833,8 +860,20 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
 
 // samp: 1, 2, 4 or 8 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
 // a standard deviation of the sample rank (50 in production).
+// One CTA of 1024 threads per SM: the CTAs of an SM that start at different times do not advance at the
+// same pace (the warp schedulers favour the older one), and with static ranges the youngest of four sets
+// the kernel's time.  The warps of one CTA are of one age, and in scan B they draw their work (items of
+// 32 * kBatch consecutive tokens) from a counter in shared memory, so they end a segment together.
+constexpr int kBandThreads = 1024;
+constexpr int kBandWarps = kBandThreads / 32;
+constexpr int kBandStage = 64;                   // list entries a warp can hold back
 template <int S>
-__global__ void __launch_bounds__(kThreads, 4)
+constexpr size_t band_smem_bytes() {             // dynamic: the warps' staging slots, one scratch row per thread
+    return (size_t)kBandWarps * kBandStage * sizeof(uint2) + (size_t)kBandThreads * S * 4;
+}
+
+template <int S>
+__global__ void __launch_bounds__(kBandThreads, 1)
 route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ cls, int64_t cls_b_stride,
                   int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int upp,
                   int k_nominal, int min_per_token, uint32_t* __restrict__ state_all,
@@ -843,22 +882,21 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                   uint32_t* __restrict__ unit_sums, uint2* __restrict__ list_all, uint32_t list_cap,
                   long long total_units, int skip_scan_a, unsigned long long wait_ns, int samp, int z_tenths) {
     constexpr int kBatch = S >= 8 ? 32 / S : 4;  // tokens in flight per thread (at most 32 score registers)
+    extern __shared__ __align__(16) uint32_t band_dyn[];
     __shared__ __align__(16) uint32_t shist[kBins13];
-    __shared__ uint32_t s_w[kWarps];
-    __shared__ uint32_t s_pick[3];
+    __shared__ uint32_t s_w[kBandWarps];
+    __shared__ uint32_t s_pick[2];
     __shared__ uint32_t s_bc[4];
     __shared__ uint32_t s_cnt[2];
+    __shared__ uint32_t s_next;
     __shared__ int s_last;
-    constexpr int kStage = 64;                   // list entries a warp can hold back
-    __shared__ uint2 s_stage[kWarps][kStage];
-    // scan B has no use for the histogram: its words hold the segment's per-unit counts and one scratch row per thread
-    constexpr int kUnitsMax = 2048;
-    static_assert(kUnitsMax + kThreads * S <= kBins13, "scan B's scratch fits the histogram");
+    // scan B has no use for the histogram: its words hold the segment's per-unit counts
+    constexpr int kUnitsMax = kBins13;
     uint32_t* s_units = shist;
-    uint32_t* s_row = shist + kUnitsMax + threadIdx.x * S;
 
-    const int tid = threadIdx.x, lane = tid & 31;
-    uint2* stage = s_stage[tid >> 5];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint2* stage = reinterpret_cast<uint2*>(band_dyn) + warp * kBandStage;
+    uint32_t* s_row = band_dyn + kBandWarps * kBandStage * 2 + tid * S;
     const long long x0 = total_units * blockIdx.x / gridDim.x;
     const long long x1 = total_units * (blockIdx.x + 1) / gridDim.x;
     const int floor_k = min_per_token ? 1 : 0;
@@ -866,8 +904,10 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
     const bool select = k_nominal > floor_k;
 
     // ---- scan A: histogram of the top 13 key bits of the sample's candidates ---------------------
+    // the CTA covers 4 * samp units at a time: thread -> (unit du of those, sampled token sidx of the unit)
     const int per_unit = kUnit / samp;               // sampled tokens per unit
     const int du = tid / per_unit, sidx = tid - du * per_unit;
+    const int group = (kBandThreads / kUnit) * samp; // units per step of a thread
 #pragma unroll 1
     for (long long x = (skip_scan_a || !select) ? x1 : x0; x < x1;) {
         const int problem = (int)(x / upp);
@@ -880,12 +920,13 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
         uint32_t* hist = hist_all + (size_t)problem * kBins13;
         const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
         const float* rows = scores + (size_t)problem * T * S;
-        for (int i = tid; i < kBins13; i += kThreads) shist[i] = 0;
+        for (int i = tid; i < kBins13; i += kBandThreads) shist[i] = 0;
+        if (tid == 0) s_cnt[0] = 0u;
         __syncthreads();
         const uint32_t shist_base = smem_u32(shist);
         uint32_t n_routed = 0;
 #pragma unroll 1
-        for (int v = u0; v < u0 + n; v += samp * kBatch) {
+        for (int v = u0; v < u0 + n; v += group * kBatch) {
             if (v * kUnit >= len) break;
             uint4 raw[kBatch][S / 4];
             bool routed[kBatch];
@@ -893,7 +934,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             for (int i = 0; i < kBatch; ++i) {           // all of the thread's loads are in flight before the first use
                 // the thread's token of unit `unit`: run (sidx / 4) of the unit's sampled runs of four tokens;
                 // the runs of a unit start every 4 * samp tokens, shifted by the unit's number
-                const int unit = v + i * samp + du;
+                const int unit = v + i * group + du;
                 const int t = unit * kUnit + ((((sidx >> 2) * samp + (unit & (samp - 1))) << 2) | (sidx & 3));
                 routed[i] = unit < u0 + n && token_class(c, t, len) == STC_CLS_ROUTED;
                 load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);
@@ -910,14 +951,14 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                 }
             }
         }
+        n_routed = __reduce_add_sync(0xFFFFFFFFu, n_routed);
+        if (lane == 0 && n_routed) atomicAdd(&s_cnt[0], n_routed);
         __syncthreads();
-        for (int i = tid; i < kBins13; i += kThreads) {
+        for (int i = tid; i < kBins13; i += kBandThreads) {
             const uint32_t v = shist[i];
             if (v) atomicAdd(hist + i, v);
         }
-        uint32_t tot;
-        block_excl_scan(n_routed, s_w, &tot);
-        if (tid == 0 && tot) atomicAdd(state + ST_NROUTEDA, tot);
+        if (tid == 0 && s_cnt[0]) atomicAdd(state + ST_NROUTEDA, s_cnt[0]);
         __threadfence();
         __syncthreads();
         if (tid == 0)
@@ -942,12 +983,12 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                 r_lo = ceilf(r + d);
             }
             if (r_hi >= 1.f) {
-                pick_digit_n<false>(hist, kBins13, kBins13 / kThreads, (uint32_t)r_hi, s_w, s_pick);
+                settle_pick<true>(hist, kBins13, kBins13 / kBandThreads, (uint32_t)r_hi, s_w, s_pick);
                 b_hi = s_pick[0];
                 __syncthreads();
             }
             if (r_lo <= (float)m_c) {
-                pick_digit_n<false>(hist, kBins13, kBins13 / kThreads, (uint32_t)r_lo, s_w, s_pick);
+                settle_pick<true>(hist, kBins13, kBins13 / kBandThreads, (uint32_t)r_lo, s_w, s_pick);
                 b_lo = s_pick[0];
                 __syncthreads();
             }
@@ -962,6 +1003,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
     }
 
     // ---- scan B: definite bits above the band, the list inside it, counts ----------------------
+    constexpr int kItemTokens = 32 * kBatch;             // a warp's item: kBatch runs of 32 consecutive tokens
 #pragma unroll 1
     for (long long x = x0; x < x1;) {
         const int problem = (int)(x / upp);
@@ -972,23 +1014,35 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
         const int len = clamp_len(seq_len, b, T);
         uint32_t* state = state_all + (size_t)problem * ST_WORDS;
         const uint8_t* c = cls ? cls + (size_t)b * cls_b_stride + (size_t)hk * cls_h_stride : nullptr;
-        uint4 raw[kBatch][S / 4];
-        int cls_of[kBatch];
         const float* rows = scores + (size_t)problem * T * S;
         uint2* list = list_all + (size_t)problem * list_cap;
-        auto load_batch = [&](int u) {
+        const int t_begin = u0 * kUnit, t_end = min((u0 + n) * kUnit, T);
+        const int items = (t_end - t_begin + kItemTokens - 1) / kItemTokens;
+
+        if (tid < 2) s_cnt[tid] = 0u;
+        if (tid == 0) s_next = 0u;
+        for (int i = tid; i < n; i += kBandThreads) s_units[i] = 0u;
+        __syncthreads();
+        uint4 raw[kBatch][S / 4];
+        int cls_of[kBatch];
+        auto grab = [&]() {                              // the warp's next item of the segment
+            uint32_t it = 0;
+            if (lane == 0) it = atomicAdd(&s_next, 1u);
+            return (int)__shfl_sync(0xFFFFFFFFu, it, 0);
+        };
+        auto load_item = [&](int item) {
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
-                const int t = (u + i) * kUnit + tid;
-                cls_of[i] = (u + i < u0 + n && t < T) ? token_class(c, t, len) : STC_CLS_DROP;
+                const int t = t_begin + item * kItemTokens + 32 * i + lane;
+                cls_of[i] = t < t_end ? token_class(c, t, len) : STC_CLS_DROP;
                 load_raw<S>(rows + (size_t)min(t, T - 1) * S, raw[i]);
             }
         };
-        load_batch(u0);                                  // in flight while the band arrives
+        int item = grab();
+        if (item < items) load_item(item);               // in flight while the band arrives
         float lo = 0.f, hi = 0.f;
         if (select) {
             if (!wait_band(state, s_bc, abort_word, wait_ns)) return;
-            if (s_bc[1] != PATH_BAND) continue;
             band_bounds(s_bc[2], s_bc[3], lo, hi);
         }
         uint32_t pend_n = 0, pend_base = 0;              // staged entries of the warp and (lane 31) their place in the list
@@ -1002,13 +1056,11 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                 pend_n = 0;
             }
         };
-        if (tid < 2) s_cnt[tid] = 0u;
-        for (int i = tid; i < n; i += kThreads) s_units[i] = 0u;
-        __syncthreads();
         uint32_t n_routed = 0, n_above = 0;
 #pragma unroll 1
-        for (int u = u0; u < u0 + n; u += kBatch) {
-            // 1. everything that needs the batch's scores: masks, counts, the list entries (to the staging slots)
+        while (item < items) {
+            const int t0 = t_begin + item * kItemTokens + lane;      // the lane's token of run 0
+            // 1. everything that needs the item's scores: masks, counts, the list entries (to the staging slots)
             uint32_t defs[kBatch], cands[kBatch], c_mine = 0;
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
@@ -1026,11 +1078,11 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             }
             // The warp's candidates go to the list in one piece.  Its place there comes from an atomic addition
             // whose answer takes a microsecond: the entries wait in the warp's staging slots and are written out
-            // one batch later, when the answer has long arrived.
+            // one item later, when the answer has long arrived.
             flush();
             const uint32_t incl = warp_incl_scan(c_mine, lane);
             const uint32_t w_total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            const bool staged = w_total <= (uint32_t)kStage;
+            const bool staged = w_total <= (uint32_t)kBandStage;
             if (w_total) {
                 uint32_t pos = incl - c_mine;
                 if (!staged) {                           // (too many for the slots: rare; wait for the place)
@@ -1039,7 +1091,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                     pos += __shfl_sync(0xFFFFFFFFu, base, 31);
                 }
                 uint2* dst = staged ? stage : list;
-                const uint32_t lim = staged ? (uint32_t)kStage : list_cap;
+                const uint32_t lim = staged ? (uint32_t)kBandStage : list_cap;
 #pragma unroll
                 for (int i = 0; i < kBatch; ++i) {
                     uint32_t m = cands[i];
@@ -1047,7 +1099,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                     // the token's scores go to the thread's scratch row, where a score can be picked by number
 #pragma unroll
                     for (int q = 0; q < S / 4; ++q) reinterpret_cast<uint4*>(s_row)[q] = raw[i][q];
-                    const uint32_t flat = (uint32_t)((u + i) * kUnit + tid) * S;
+                    const uint32_t flat = (uint32_t)(t0 + 32 * i) * S;
                     while (m) {
                         const int j = __ffs(m) - 1;
                         m &= m - 1;
@@ -1056,8 +1108,9 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                     }
                 }
             }
-            // 2. the scores are no longer needed: the next batch's loads go out now and fly during the rest
-            if (u + kBatch < u0 + n) load_batch(u + kBatch);
+            // 2. the scores are no longer needed: the next item's loads go out now and fly during the rest
+            const int next = grab();
+            if (next < items) load_item(next);
             // 3. what only needs the masks
             if (w_total && staged) {
                 if (lane == 31) pend_base = atomicAdd(state + ST_LISTN, w_total);
@@ -1065,15 +1118,18 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             }
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
-                if (u + i < u0 + n && (u + i) * kUnit + tid < T) {
-                    const size_t at = (size_t)problem * T + (size_t)(u + i) * kUnit + tid;
-                    v_mask[at] = (uint16_t)defs[i];
-                    tie_all[at] = 0;
+                const int t = t0 + 32 * i;
+                if (t < t_end) {
+                    v_mask[(size_t)problem * T + t] = (uint16_t)defs[i];
+                    tie_all[(size_t)problem * T + t] = 0;
                 }
-                // per-unit count of definite bits, gathered in shared memory for the whole segment
+                // per-unit count of definite bits (the 32 tokens of a run lie in one unit), gathered in shared
+                // memory for the whole segment
                 const uint32_t cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(defs[i]));
-                if (lane == 0 && cnt && u + i < u0 + n) atomicAdd(&s_units[u + i - u0], cnt);
+                const int run_t = t0 - lane + 32 * i;
+                if (lane == 0 && cnt && run_t < t_end) atomicAdd(&s_units[run_t / kUnit - u0], cnt);
             }
+            item = next;
         }
         flush();
         n_routed = __reduce_add_sync(0xFFFFFFFFu, n_routed);
@@ -1085,7 +1141,7 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
             if (s_cnt[1]) atomicAdd(state + ST_ABOVE, s_cnt[1]);
         }
         // (plain stores: the settle kernel, which runs after this one, adds the listed pairs it keeps)
-        for (int i = tid; i < n; i += kThreads) unit_sums[(size_t)problem * upp + u0 + i] = s_units[i];
+        for (int i = tid; i < n; i += kBandThreads) unit_sums[(size_t)problem * upp + u0 + i] = s_units[i];
         __syncthreads();                                 // the scratch is reused by the next segment
     }
 }
@@ -1306,7 +1362,8 @@ size_t route_ws_bytes(const Geom& g) { return carve(g, nullptr).total_bytes; }
 namespace {
 
 // CTAs of a cooperatively launched kernel that can be resident at once.
-cudaError_t coop_grid_limit(const void* fn, std::atomic<int>* cached /*[kMaxDevices]*/, int* limit) {
+cudaError_t coop_grid_limit(const void* fn, int threads, size_t dyn_smem, std::atomic<int>* cached /*[kMaxDevices]*/,
+                            int* limit) {
     // per device: the occupancy of a kernel is a property of the kernel and the device, the
     // query is cheap next to a cooperative launch, and a process may drive several devices
     constexpr int kMaxDevices = 64;
@@ -1317,7 +1374,7 @@ cudaError_t coop_grid_limit(const void* fn, std::atomic<int>* cached /*[kMaxDevi
     if (v == 0) {
         int sms = 0, per_sm = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, 0);
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, dyn_smem);
         if (e != cudaSuccess) return e;
         if (sms <= 0 || per_sm <= 0) return cudaErrorLaunchOutOfResources;
         v = sms * per_sm;
@@ -1358,7 +1415,11 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
     cudaError_t e;
     int limit = 0;
     if (band) {
-        e = coop_grid_limit(reinterpret_cast<const void*>(route_band_kernel<S>), cached_band, &limit);
+        e = cudaFuncSetAttribute(route_band_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)band_smem_bytes<S>());
+        if (e != cudaSuccess) return e;
+        e = coop_grid_limit(reinterpret_cast<const void*>(route_band_kernel<S>), kBandThreads, band_smem_bytes<S>(),
+                            cached_band, &limit);
         if (e != cudaSuccess) return e;
         const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
         int skip_scan_a = knob == 4;
@@ -1369,8 +1430,8 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
         void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token,
                         &state, &hist13, &abort_word, &v_mask, &tie, &unit_sums, &list, &list_cap, &total_units,
                         &skip_scan_a, &wait_ns, &samp, &z_tenths};
-        e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_band_kernel<S>), dim3(grid), dim3(kThreads),
-                                        args, 0, st);
+        e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_band_kernel<S>), dim3(grid),
+                                        dim3(kBandThreads), args, band_smem_bytes<S>(), st);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(route_settle_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSettleSmem);
         if (e != cudaSuccess) return e;
@@ -1379,7 +1440,7 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    e = coop_grid_limit(reinterpret_cast<const void*>(route_select_kernel<S>), cached_select, &limit);
+    e = coop_grid_limit(reinterpret_cast<const void*>(route_select_kernel<S>), kThreads, 0, cached_select, &limit);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
     int first_pass = (knob >= 1 && knob <= 3) ? knob : 0;
