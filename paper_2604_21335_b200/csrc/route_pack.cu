@@ -6,7 +6,7 @@
 // the lower flat index.  `take` depends on the routed-token count, which only
 // the device knows, so everything is resolved on the device:
 //
-//   GLOBAL budget, score arrays of at least twice the L2 size: the band kernel and the
+//   GLOBAL budget, score arrays from half the L2 size on: the band kernel and the
 //   settle kernel (described where they are defined, further down) find the threshold in
 //   one scan of the scores plus a sampled one; the multi-pass kernel below then only
 //   redoes the problems they could not settle.  Otherwise:
@@ -767,6 +767,8 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
     __shared__ uint32_t shist[2048];
     __shared__ uint32_t s_w[kSettleWarps];
     __shared__ uint32_t s_pick[2];
+    __shared__ uint32_t s_ntie;
+    constexpr int kTieRankMax = 4096;                    // pairs on the threshold that are ranked here (all-pairs count)
     const int tid = threadIdx.x;
     const int problem = blockIdx.x;
     uint32_t* state = state_all + (size_t)problem * ST_WORDS;
@@ -789,7 +791,6 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
     const uint2* list = list_all + (size_t)problem * list_cap;
     const bool word_ok = (reinterpret_cast<uintptr_t>(v_mask) & 3u) == 0 && (T & 1) == 0;
     uint16_t* mask_row = v_mask + (size_t)problem * T;
-    uint16_t* tie_row = tie_all + (size_t)problem * T;
     uint32_t* sums_row = unit_sums + (size_t)problem * upp;
     constexpr int kInFlight = 8;                         // list entries a thread has in flight
     const bool staged = n_list <= (uint32_t)kSettleKeys;
@@ -830,7 +831,15 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
     // the per-unit counts of what is added are gathered in the histogram's words when the problem's units fit there
     const bool local_sums = upp <= 2048;
     if (local_sums) for (int i = tid; i < upp; i += kSettleThreads) shist[i] = 0u;
+    if (tid == 0) s_ntie = 0u;
+    uint32_t* s_ties = s_keys;                           // (the staged keys have served)
     __syncthreads();
+    auto keep = [&](uint32_t flat) {                     // the pair's definite bit and its unit's count
+        const uint32_t t = flat / S, j = flat - t * S;
+        or16(mask_row + t, 1u << j, word_ok);
+        if (local_sums) atomicAdd(&shist[t / kUnit], 1u);
+        else atomicAdd(sums_row + t / kUnit, 1u);
+    };
 #pragma unroll 1
     for (uint32_t e0 = tid; e0 < n_list; e0 += kInFlight * kSettleThreads) {
         uint2 en[kInFlight];
@@ -840,13 +849,33 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
         for (int i = 0; i < kInFlight; ++i) {
             const uint32_t key = float_key(__uint_as_float(en[i].x));
             if (e0 + i * kSettleThreads >= n_list || key < tau) continue;
-            const uint32_t t = en[i].y / S, j = en[i].y - t * S;
-            if (t >= (uint32_t)T) continue;              // (cannot happen: the scan wrote the entry)
-            const uint32_t add = key > tau ? 1u : 1u << 16;
-            or16((key > tau ? mask_row : tie_row) + t, 1u << j, word_ok);
-            if (local_sums) atomicAdd(&shist[t / kUnit], add);
-            else atomicAdd(sums_row + t / kUnit, add);
+            if (en[i].y / S >= (uint32_t)T) continue;    // (cannot happen: the scan wrote the entry)
+            if (key > tau) {
+                keep(en[i].y);
+            } else {                                     // on the threshold: settled below, in flat-index order
+                const uint32_t at = atomicAdd(&s_ntie, 1u);
+                if (at < (uint32_t)kSettleKeys) s_ties[at] = en[i].y;
+            }
         }
+    }
+    __syncthreads();
+    // The pairs on the threshold: the krem lowest flat indices are kept.  (A problem's tie array is not
+    // used after this kernel -- the compaction does not read it for a settled problem -- so the scan did
+    // not have to clear it.)
+    const uint32_t n_tie = s_ntie;
+    if (n_tie > (uint32_t)kSettleKeys || (krem < n_tie && n_tie > (uint32_t)kTieRankMax)) {   // massive ties: the multi-pass kernel redoes the problem
+        if (tid == 0) {
+            state[ST_PATH] = PATH_WIDE;
+            atomicExch(abort_word + 1, 1u);
+        }
+        return;
+    }
+    for (uint32_t e = tid; e < n_tie; e += kSettleThreads) {
+        const uint32_t flat = s_ties[e];
+        uint32_t rank = 0;
+        if (krem < n_tie)
+            for (uint32_t o = 0; o < n_tie; ++o) rank += s_ties[o] < flat;
+        if (rank < krem) keep(flat);
     }
     if (local_sums) {
         __syncthreads();
@@ -855,7 +884,7 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
             if (v) sums_row[i] += v;
         }
     }
-    if (tid == 0) { state[ST_FLAGS] = 0u; state[ST_PREFIX] = tau; state[ST_KREM] = krem; }
+    if (tid == 0) { state[ST_FLAGS] = 0u; state[ST_PREFIX] = tau; state[ST_KREM] = 0u; }
 }
 
 // samp: 1, 2, 4 or 8 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
@@ -1121,7 +1150,6 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                 const int t = t0 + 32 * i;
                 if (t < t_end) {
                     v_mask[(size_t)problem * T + t] = (uint16_t)defs[i];
-                    tie_all[(size_t)problem * T + t] = 0;
                 }
                 // per-unit count of definite bits (the 32 tokens of a run lie in one unit), gathered in shared
                 // memory for the whole segment
@@ -1267,10 +1295,12 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
     if (t_begin >= len && !owns_end) return;
 
     uint32_t krem = 0, flags = 0;
+    bool use_tie = true;                        // a problem settled by the band path has no tie bits (and no cleared tie array)
     if (mode == STC_MODE_GLOBAL) {
         const uint32_t* state = state_all + (size_t)problem * ST_WORDS;
         flags = __ldcg(state + ST_FLAGS);
         krem = flags ? 0u : __ldcg(state + ST_KREM);
+        use_tie = __ldcg(state + ST_PATH) != PATH_BAND;
     }
     // base counts from the preceding units
     uint32_t bd = 0, be = 0;
@@ -1290,7 +1320,7 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
     for (int i = 0; i < kTokPerThread; ++i) {
         const int t = t0 + i;
         def[i] = t < len ? v_mask[(size_t)problem * T + t] : 0u;
-        tie[i] = t < len ? tie_all[(size_t)problem * T + t] : 0u;
+        tie[i] = (t < len && use_tie) ? tie_all[(size_t)problem * T + t] : 0u;
         nd += __popc(def[i]);
         ne += __popc(tie[i]);
     }
@@ -1403,12 +1433,13 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
     // it left (it returns at once when there is none) and does everything in PER_TOKEN mode.
     // (a floor of one group per token with a nominal budget of none is the budget error: the multi-pass kernel reports it)
     // It pays when the scores do not stay in L2 between the scans (each of the four passes of the multi-pass
-    // kernel is then a trip to HBM); smaller score arrays are quicker with the multi-pass kernel.
+    // kernel is then a trip to HBM): measured, from about half the L2 size on; smaller score arrays
+    // are as quick or quicker with the multi-pass kernel.
     bool big = false;
     {
         int dev = 0, l2 = 0;
         if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) == cudaSuccess)
-            big = (double)g.problems * g.T * g.S * 4.0 >= 2.0 * (double)l2;
+            big = (double)g.problems * g.T * g.S * 4.0 >= 0.5 * (double)l2;
     }
     const bool band = mode == STC_MODE_GLOBAL && ((knob == 0 && big) || knob >= 4) &&
                       !(min_per_token && k_nominal == 0);
@@ -1510,7 +1541,7 @@ void set_route_select_knobs(int first_pass, unsigned long long wait_ns) {
 }  // namespace stc
 
 // Test hook, not part of the public interface (not declared in stc.h).  first_pass: 0 = normal (for score
-// arrays well beyond the L2 size the band kernel, then the multi-pass kernel for what it left; else the
+// arrays of half the L2 size and beyond the band kernel, then the multi-pass kernel for what it left; else the
 // multi-pass kernel alone); -1 = the multi-pass kernel alone; 1..3 = the
 // multi-pass kernel alone, starting at that histogram pass; 4 = the band kernel without its first scan;
 // 5 = the band kernel with every token in its sample (the band is then exact); 6 = the band kernel with

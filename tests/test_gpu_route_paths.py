@@ -5,8 +5,8 @@ around the threshold, one full scan lists the pairs inside it and counts the pai
 count check accepts or rejects the band) and the multi-pass radix kernel, which also takes over the
 problems whose band was rejected or whose list overflowed.  A test-only launch parameter (not in the
 public header) selects among them; the result must not depend on it.
-   0  production: the band kernel for score arrays well beyond the L2 size (then the multi-pass kernel for
-      what it left), the multi-pass kernel alone for smaller ones
+   0  production: the band kernel for score arrays of half the L2 size and beyond (then the multi-pass kernel
+      for what it left), the multi-pass kernel alone for smaller ones
    7  the production band kernel whatever the size
   -1  multi-pass kernel alone
    5  band kernel with every token in the sample (the band is exact)
@@ -72,6 +72,24 @@ def test_massive_ties_and_skewed_scores(knob):
     o = H.oracle_pipeline(w, d)
     try:
         knobs(knob)
+        g = H.gpu_pipeline(w, d)
+        torch.cuda.synchronize()
+    finally:
+        knobs(0)
+    H.assert_bit_exact_write_side(w, g, o)
+
+
+@pytest.mark.parametrize("step", [4096.0, 256.0, 32.0])
+def test_ties_on_the_threshold_inside_the_band(step):
+    """Scores on a grid: with 4096 steps per unit a few dozen pairs share the threshold value, with 256 several
+    hundred (both ranked by flat index in the settle kernel), with 32 several thousand (too many to rank there:
+    the multi-pass kernel redoes the problem)."""
+    w = W.shrink(W.get("cfg1"), n_q_heads=2, n_kv_heads=2, t_cache=40000, token_budget=512)
+    d = W.make_inputs(w, DEV)
+    d["scores"] = torch.round(d["scores"] * step) / step
+    o = H.oracle_pipeline(w, d)
+    try:
+        knobs(7)
         g = H.gpu_pipeline(w, d)
         torch.cuda.synchronize()
     finally:
