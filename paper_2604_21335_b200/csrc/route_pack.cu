@@ -550,10 +550,12 @@ route_select_kernel(const float* __restrict__ scores, const uint8_t* __restrict_
 //   pairs counted above the band, the take-th largest candidate is the (take - above)-th largest of
 //   the list, provided above < take <= above + list length -- which is the check that the band was
 //   right.  Radix select over the list, then one pass that sets the definite bit of every listed pair
-//   above the threshold and the tie bit of every pair on it (the compaction resolves ties in
-//   flat-index order, as after the multi-pass kernel).
+//   above the threshold; the pairs on the threshold are ranked by flat index and the lowest are kept
+//   (the rule the compaction applies to the tie bits of the multi-pass kernel), so a settled problem
+//   has no tie bits and its part of the tie array is neither cleared nor read.
 // A problem whose band was wrong, or holds more pairs than the list has room for (massive ties), is
-// marked PATH_WIDE and left to the multi-pass kernel that runs next; the result is the same either way.
+// or has more than a few thousand pairs on the threshold, is marked PATH_WIDE and left to the multi-pass
+// kernel that runs next; the result is the same either way.
 
 template <bool kSharedHist>
 __device__ void pick_digit_n(const uint32_t* __restrict__ hist, int nbins, int per, uint32_t krem,
@@ -708,7 +710,7 @@ __device__ __forceinline__ void band_token(const uint4 (&raw)[S / 4], bool selec
 // Checks the band (above < take <= above + list length), finds the (take - above)-th largest key of the
 // list by radix select (11 + 11 + 10 bits; the keys are staged in shared memory when they fit, else every
 // pass reads the list, which sits in L2), then sets the definite bit of every listed pair above the
-// threshold and the tie bit of every pair on it, and adds them to the per-unit counts.
+// threshold and of the lowest-indexed pairs on it, and adds them to the per-unit counts.
 constexpr int kSettleThreads = 1024;
 constexpr int kSettleWarps = kSettleThreads / 32;
 constexpr int kSettleKeys = 45056;                 // keys staged in shared memory (176 KiB)
@@ -761,8 +763,7 @@ template <int S>
 __global__ void __launch_bounds__(kSettleThreads, 1)
 route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abort_word,
                     const uint2* __restrict__ list_all, uint32_t list_cap, uint16_t* __restrict__ v_mask,
-                    uint16_t* __restrict__ tie_all, uint32_t* __restrict__ unit_sums, int T, int upp,
-                    int k_nominal, int min_per_token) {
+                    uint32_t* __restrict__ unit_sums, int T, int upp, int k_nominal, int min_per_token) {
     extern __shared__ __align__(16) uint32_t s_keys[];
     __shared__ uint32_t shist[2048];
     __shared__ uint32_t s_w[kSettleWarps];
@@ -907,9 +908,9 @@ route_band_kernel(const float* __restrict__ scores, const uint8_t* __restrict__ 
                   int64_t cls_h_stride, const int32_t* __restrict__ seq_len, int Hkv, int T, int upp,
                   int k_nominal, int min_per_token, uint32_t* __restrict__ state_all,
                   uint32_t* __restrict__ hist_all, uint32_t* __restrict__ abort_word,
-                  uint16_t* __restrict__ v_mask, uint16_t* __restrict__ tie_all,
-                  uint32_t* __restrict__ unit_sums, uint2* __restrict__ list_all, uint32_t list_cap,
-                  long long total_units, int skip_scan_a, unsigned long long wait_ns, int samp, int z_tenths) {
+                  uint16_t* __restrict__ v_mask, uint32_t* __restrict__ unit_sums, uint2* __restrict__ list_all,
+                  uint32_t list_cap, long long total_units, int skip_scan_a, unsigned long long wait_ns, int samp,
+                  int z_tenths) {
     constexpr int kBatch = S >= 8 ? 32 / S : 4;  // tokens in flight per thread (at most 32 score registers)
     extern __shared__ __align__(16) uint32_t band_dyn[];
     __shared__ __align__(16) uint32_t shist[kBins13];
@@ -1459,7 +1460,7 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
         int samp = knob == 5 ? 1 : (keys >= (1 << 20) ? 8 : keys >= (1 << 19) ? 4 : keys >= (1 << 18) ? 2 : 1);
         int z_tenths = knob == 6 ? 0 : 50;
         void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token,
-                        &state, &hist13, &abort_word, &v_mask, &tie, &unit_sums, &list, &list_cap, &total_units,
+                        &state, &hist13, &abort_word, &v_mask, &unit_sums, &list, &list_cap, &total_units,
                         &skip_scan_a, &wait_ns, &samp, &z_tenths};
         e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(route_band_kernel<S>), dim3(grid),
                                         dim3(kBandThreads), args, band_smem_bytes<S>(), st);
@@ -1467,7 +1468,7 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
         e = cudaFuncSetAttribute(route_settle_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSettleSmem);
         if (e != cudaSuccess) return e;
         route_settle_kernel<S><<<(unsigned)g.problems, kSettleThreads, kSettleSmem, st>>>(
-            state, abort_word, list, list_cap, v_mask, tie, unit_sums, T, upp, k_nominal, min_per_token);
+            state, abort_word, list, list_cap, v_mask, unit_sums, T, upp, k_nominal, min_per_token);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
