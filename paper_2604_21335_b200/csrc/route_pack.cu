@@ -888,7 +888,7 @@ route_settle_kernel(uint32_t* __restrict__ state_all, uint32_t* __restrict__ abo
     if (tid == 0) { state[ST_FLAGS] = 0u; state[ST_PREFIX] = tau; state[ST_KREM] = 0u; }
 }
 
-// samp: 1, 2, 4 or 8 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
+// samp: a power of two up to 16 -- scan A looks at one token in `samp`.  z_tenths: the band's half-width in tenths of
 // a standard deviation of the sample rank (50 in production).
 // One CTA of 1024 threads per SM: the CTAs of an SM that start at different times do not advance at the
 // same pace (the warp schedulers favour the older one), and with static ranges the youngest of four sets
@@ -1455,9 +1455,9 @@ cudaError_t launch_select(const Geom& g, const float* scores, const uint8_t* cls
         if (e != cudaSuccess) return e;
         const unsigned grid = (unsigned)(total_units < limit ? total_units : limit);
         int skip_scan_a = knob == 4;
-        // scan A samples one token in `samp`, keeping at least 2^17 keys of a problem in the sample
+        // scan A samples one token in `samp`, keeping at least 2^16 keys of a problem in the sample
         const long long keys = (long long)g.T * g.S;
-        int samp = knob == 5 ? 1 : (keys >= (1 << 20) ? 8 : keys >= (1 << 19) ? 4 : keys >= (1 << 18) ? 2 : 1);
+        int samp = knob == 5 ? 1 : (keys >= (1 << 20) ? 16 : keys >= (1 << 19) ? 8 : keys >= (1 << 18) ? 4 : keys >= (1 << 17) ? 2 : 1);
         int z_tenths = knob == 6 ? 0 : 50;
         void* args[] = {&scores, &cls, &cls_b, &cls_h, &seq_len, &Hkv, &T, &upp, &k_nominal, &min_per_token,
                         &state, &hist13, &abort_word, &v_mask, &unit_sums, &list, &list_cap, &total_units,
