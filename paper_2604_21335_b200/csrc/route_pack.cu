@@ -1296,12 +1296,10 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
     if (t_begin >= len && !owns_end) return;
 
     uint32_t krem = 0, flags = 0;
-    bool use_tie = true;                        // a problem settled by the band path has no tie bits (and no cleared tie array)
     if (mode == STC_MODE_GLOBAL) {
         const uint32_t* state = state_all + (size_t)problem * ST_WORDS;
         flags = __ldcg(state + ST_FLAGS);
         krem = flags ? 0u : __ldcg(state + ST_KREM);
-        use_tie = __ldcg(state + ST_PATH) != PATH_BAND;
     }
     // base counts from the preceding units
     uint32_t bd = 0, be = 0;
@@ -1321,7 +1319,10 @@ route_compact_kernel(const uint4* __restrict__ v, const int32_t* __restrict__ se
     for (int i = 0; i < kTokPerThread; ++i) {
         const int t = t0 + i;
         def[i] = t < len ? v_mask[(size_t)problem * T + t] : 0u;
-        tie[i] = (t < len && use_tie) ? tie_all[(size_t)problem * T + t] : 0u;
+        tie[i] = t < len ? tie_all[(size_t)problem * T + t] : 0u;
+        // a problem settled by the band path has no tie bits, no cleared tie array and a remaining rank of zero:
+        // whatever was read there is dropped
+        tie[i] = krem ? tie[i] : 0u;
         nd += __popc(def[i]);
         ne += __popc(tie[i]);
     }
