@@ -658,8 +658,8 @@ __device__ __forceinline__ bool wait_band(const uint32_t* state, uint32_t* s_bc,
 // The scores whose 13-bit digit lies in [b_lo, b_hi], as a closed float interval (scores are not NaN).
 __device__ __forceinline__ void band_bounds(uint32_t b_lo, uint32_t b_hi, float& lo, float& hi) {
     uint32_t klo = b_lo << kShift13, khi = (b_hi << kShift13) | ((1u << kShift13) - 1u);
-    klo = max(klo, 0x007FFFFFu);                   // -inf
-    khi = min(khi, 0xFF800000u);                   // +inf
+    klo = max(klo, 0x00800000u);                   // -FLT_MAX: the edges stay finite (band_token subtracts them), and an
+    khi = min(khi, 0xFF7FFFFFu);                   // +FLT_MAX  infinite score is then simply below or above the band
     if (khi == 0x7FFFFFFFu) khi = 0x7FFFFFFEu;     // the key of -0 is unused: stop below zero
     lo = key_float(klo);
     hi = key_float(khi);
@@ -684,13 +684,20 @@ __device__ __forceinline__ void band_token(const uint4 (&raw)[S / 4], bool selec
     def = 0;
     cand = 0;
     if (select) {
-        uint32_t ge = 0;
+        // x > hi  <=>  hi - x is negative, x >= lo  <=>  x - lo is not (a difference of two different floats is
+        // never zero without flush-to-zero, which this library is not built with; equal floats give +0): the
+        // subtractions run on the FMA pipe, which the scan leaves idle, and one funnel shift per score moves the
+        // sign into the mask, instead of compare + select + or on the pipe the scan is bound by.  The edges are
+        // finite (band_bounds), so an infinite score is simply above or below the band.
+        uint32_t above = 0, below = 0;
 #pragma unroll
-        for (int j = 0; j < S; ++j) {
-            def |= (x[j] > hi ? 1u : 0u) << j;
-            ge |= (x[j] >= lo ? 1u : 0u) << j;
+        for (int j = S - 1; j >= 0; --j) {
+            const float xj = __fadd_rn(x[j], 0.f);   // -0 -> +0, as in the keys (-0 - +0 would be -0)
+            above = __funnelshift_l(__float_as_uint(__fsub_rn(hi, xj)), above, 1);
+            below = __funnelshift_l(__float_as_uint(__fsub_rn(xj, lo)), below, 1);
         }
-        cand = ge & ~def;
+        def = above;
+        cand = ~below & ~above & ((1u << S) - 1u);
     }
     if (min_per_token && def == 0u) {
         float bx = x[0];

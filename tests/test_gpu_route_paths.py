@@ -97,6 +97,35 @@ def test_ties_on_the_threshold_inside_the_band(step):
     H.assert_bit_exact_write_side(w, g, o)
 
 
+@pytest.mark.parametrize("knob", [7, 5, -1])
+def test_signed_zeros_and_infinities_around_the_threshold(knob):
+    """The scores are shifted so that the budget's threshold is zero, then sprinkled with +0, -0 (equal as keys),
+    +inf and -inf: the band's edges sit next to zero, the pairs on the threshold carry both signs of zero."""
+    w = W.shrink(W.get("cfg1"), n_q_heads=2, n_kv_heads=2, t_cache=40000, token_budget=512)
+    d = W.make_inputs(w, DEV)
+    s = d["scores"]
+    T, S, K = w.t_cache, w.n_groups, w.k_nominal
+    gen = torch.Generator(device="cpu").manual_seed(5)
+    for h in range(2):
+        rest = torch.sort(s[0, h], dim=1, descending=True).values[:, 1:].reshape(-1)   # all but each token's maximum
+        kth = torch.topk(rest, T * (K - 1)).values[-1]
+        s[0, h] -= kth                                       # the (N K - N)-th largest remaining score is now +0
+        flat = s[0, h].view(-1)
+        idx = torch.randperm(T * S, generator=gen)[:1200].to(flat.device)
+        flat[idx[:300]] = 0.0
+        flat[idx[300:600]] = -0.0
+        flat[idx[600:900]] = float("inf")
+        flat[idx[900:]] = float("-inf")
+    o = H.oracle_pipeline(w, d)
+    try:
+        knobs(knob)
+        g = H.gpu_pipeline(w, d)
+        torch.cuda.synchronize()
+    finally:
+        knobs(0)
+    H.assert_bit_exact_write_side(w, g, o)
+
+
 def test_band_kernel_wait_expires_in_an_orderly_way():
     """Without its first scan nobody publishes a band, so every wait of the band kernel runs into its limit."""
     w = W.shrink(W.get("cfg1"), n_q_heads=4, n_kv_heads=4, t_cache=6000)
