@@ -624,7 +624,7 @@ def run_gpu(args, r: D.Rank):
 
 KERNEL_OF = {"page_meta": "page_meta_kernel", "quest_select": "quest_select_kernel",   # (or quest_filter_kernel, see below)
              "decode_attn": "decode_attn_kernel", "pack_values": "route_compact_kernel",
-             "route_mask": "route_select_kernel"}
+             "route_mask": "route_band_kernel"}   # (route_select_kernel below half the L2 size of scores; never the step's dominant call)
 
 # Per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes) of the step's dominant
 # kernel from the committed ncu captures under profiles/, keyed by (workload, batch, budget, keep, call);
