@@ -22,6 +22,9 @@
  *     (budget too small for the routed-token count, packed-capacity overflow)
  *     are written to a caller-provided per-problem status array; kernels never
  *     trap and never read or write out of bounds because of them.
+ *   - k, v, kmin, kmax, q, scores, v_packed and out must start on 16-byte
+ *     boundaries (the kernels move them in 16-byte pieces); a call given one
+ *     that does not returns STC_ERR_INVALID_ARG.
  *   - head_dim must be 128, page_size 16, n_groups in {4, 8, 16},
  *     n_q_heads a multiple of n_kv_heads with at most 8 query heads per KV head.
  *

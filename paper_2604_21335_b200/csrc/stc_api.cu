@@ -43,6 +43,12 @@ struct Range {
 
 }  // namespace
 
+namespace {
+// The kernels move keys, values, queries, page metadata and scores in 16-byte pieces.
+template <typename... P>
+bool aligned16(P... p) { return ((reinterpret_cast<uintptr_t>(p) | ...) & 15u) == 0; }
+}  // namespace
+
 extern "C" {
 
 const char* stc_status_string(int32_t status) {
@@ -89,6 +95,7 @@ int32_t stc_build_page_meta(const stc_shape* shape, const stc_cache* cache, int3
     if (!cache) return STC_ERR_INVALID_ARG;
     if (empty(g)) return STC_OK;
     if (!cache->k || !cache->kmin || !cache->kmax || page_begin < 0) return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->k, cache->kmin, cache->kmax)) return STC_ERR_INVALID_ARG;
     return cuda_rc(launch_page_meta(g, cache->k, cache->kmin, cache->kmax, page_begin, page_end,
                                     static_cast<cudaStream_t>(stream)));
 }
@@ -112,6 +119,7 @@ int32_t stc_quest_select_window(const stc_shape* shape, const stc_cache* cache, 
     if (!cache || token_budget < 0 || max_pages < 0 || n_recent_pages < 0) return STC_ERR_INVALID_ARG;
     if (empty(g)) return STC_OK;
     if (!cache->kmin || !cache->kmax || !q || !page_ids || !n_pages) return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->kmin, cache->kmax, q)) return STC_ERR_INVALID_ARG;
     const int want = token_budget / kPage < g.P ? token_budget / kPage : g.P;
     if (max_pages < want) return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, select_ws_bytes(g));
@@ -149,7 +157,8 @@ int32_t route_pack_phases(const stc_shape* shape, const void* v, const float* sc
     if (class_head_stride != 0 && class_head_stride != g.T) return STC_ERR_INVALID_ARG;
     if (empty(g)) return STC_OK;
     if (!out->v_mask) return STC_ERR_INVALID_ARG;
-    if ((phases & 1) && !scores) return STC_ERR_INVALID_ARG;
+    if ((phases & 1) && (!scores || !aligned16(scores))) return STC_ERR_INVALID_ARG;
+    if ((phases & 2) && !aligned16(v, out->v_packed)) return STC_ERR_INVALID_ARG;
     if ((phases & 2) && (!v || !out->v_packed || !out->v_offs || !total_groups || !status || out->cap_groups < 0))
         return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, route_ws_bytes(g));
@@ -229,6 +238,7 @@ int32_t stc_append_tokens(const stc_shape* shape, const stc_cache* cache, const 
     if (!cache->k || !cache->kmin || !cache->kmax || !cache->v_packed || !cache->v_mask || !cache->v_offs ||
         cache->cap_groups < 0 || !v || !old_len || !total_groups || !status)
         return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->k, cache->kmin, cache->kmax, cache->v_packed, v)) return STC_ERR_INVALID_ARG;
     return cuda_rc(launch_append(g, cache->k, cache->kmin, cache->kmax, v, old_len, max_new, cache->v_packed,
                                  cache->v_mask, cache->v_offs, cache->cap_groups, total_groups, status,
                                  static_cast<cudaStream_t>(stream)));
@@ -248,6 +258,7 @@ int32_t stc_route_new_pages(const stc_shape* shape, const stc_cache* cache, cons
     if (!cache->v_packed || !cache->v_mask || !cache->v_offs || cache->cap_groups < 0 || !scores || !first_page ||
         !total_groups || !status)
         return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->v_packed, scores)) return STC_ERR_INVALID_ARG;
     return cuda_rc(launch_route_new_pages(g, scores, first_page, k_nominal, min_per_token, mode, cache->v_packed,
                                           cache->v_mask, cache->v_offs, cache->cap_groups, total_groups, status,
                                           static_cast<cudaStream_t>(stream)));
@@ -269,8 +280,7 @@ int32_t stc_decode_attn(const stc_shape* shape, const stc_cache* cache, const vo
     if (max_pages > g.P && !page_ids) return STC_ERR_INVALID_ARG;
     if (g.T > 0 && (!cache->k || !cache->v_packed || !cache->v_mask || !cache->v_offs || cache->cap_groups < 0))
         return STC_ERR_INVALID_ARG;
-    if (((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v_packed)) & 15u) != 0)
-        return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->k, cache->v_packed, q, out)) return STC_ERR_INVALID_ARG;
     rc = check_ws(ws, ws_bytes, attn_ws_bytes(g, max_pages));
     if (rc != STC_OK) return rc;
     return cuda_rc(launch_decode_attn(g, cache->k, cache->v_packed, cache->v_mask, cache->v_offs,
@@ -299,8 +309,7 @@ int32_t stc_decode_step(const stc_shape* shape, const stc_cache* cache, const vo
     if (!cache->kmin || !cache->kmax || !cache->k || !cache->v_packed || !cache->v_mask || !cache->v_offs ||
         cache->cap_groups < 0)
         return STC_ERR_INVALID_ARG;
-    if (((reinterpret_cast<uintptr_t>(cache->k) | reinterpret_cast<uintptr_t>(cache->v_packed)) & 15u) != 0)
-        return STC_ERR_INVALID_ARG;
+    if (!aligned16(cache->k, cache->v_packed, cache->kmin, cache->kmax, q, out)) return STC_ERR_INVALID_ARG;
     const int want = token_budget / kPage < g.P ? token_budget / kPage : g.P;
     if (max_pages < want || max_pages > g.P) return STC_ERR_INVALID_ARG;
     rc = check_ws(ws_select, ws_select_bytes, select_ws_bytes(g));

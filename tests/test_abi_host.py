@@ -78,6 +78,15 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     assert lib.stc_quest_select(C.byref(cs), C.byref(cc), fake, 1024, 64, fake, fake, None, fake, 16, st) == 3
     assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, None, 64, 0.1, fake, None, fake, 1 << 30, st) == 1
     assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, fake, 64, 0.1, fake, None, fake, 16, st) == 3
+    # tensors the kernels move in 16-byte pieces must start on 16-byte boundaries
+    odd = C.c_void_p(0x1008)
+    assert lib.stc_quest_select(C.byref(cs), C.byref(cc), odd, 1024, 64, fake, fake, None, fake, 1 << 30, st) == 1
+    assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), odd, fake, fake, 64, 0.1, fake, None, fake, 1 << 30, st) == 1
+    assert lib.stc_decode_attn(C.byref(cs), C.byref(cc), fake, fake, fake, 64, 0.1, odd, None, fake, 1 << 30, st) == 1
+    assert lib.stc_route_pack(C.byref(cs), fake, odd, None, 0, 4, 1, 0, C.byref(cc), fake, fake, fake, 1 << 30, st) == 1
+    assert lib.stc_route_pack(C.byref(cs), odd, fake, None, 0, 4, 1, 0, C.byref(cc), fake, fake, fake, 1 << 30, st) == 1
+    cc_odd = Bd._Cache(odd, fake, fake, fake, fake, fake, 100)
+    assert lib.stc_build_page_meta(C.byref(cs), C.byref(cc_odd), 0, -1, st) == 1
     # the window variant: a negative window is an argument error, a valid one reaches the workspace check
     assert lib.stc_quest_select_window(C.byref(cs), C.byref(cc), fake, 1024, -1, 64, fake, fake, None, fake, 1 << 30, st) == 1
     assert lib.stc_quest_select_window(C.byref(cs), C.byref(cc), fake, 1024, 4, 64, fake, fake, None, None, 0, st) == 3
