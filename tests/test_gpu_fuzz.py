@@ -2,13 +2,17 @@
 token to a dozen thousand (both selection kernels, CTA ranges inside and across problems),
 ragged and empty sequences, class mixes, both routing modes, budgets from zero to all groups,
 continuous and heavily tied scores.  Every case against the CPU checker: integer outputs bit
-for bit, attention within the stated tolerance."""
+for bit, attention within the stated tolerance.  Each seed runs twice: with the routing selection
+kernel the library would pick for the size (the multi-pass kernel at these sizes) and with the band
+kernel forced through the library's test-only launch parameter."""
+import ctypes as C
 import random
 
 import numpy as np
 import pytest
 import torch
 
+import paper_2604_21335_b200 as P
 from paper_2604_21335_b200 import workload as W
 
 import helpers as H
@@ -17,8 +21,24 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+def knobs(first_pass):
+    lib = P.load_library()
+    lib.stc_test_route_select_knobs.restype = None
+    lib.stc_test_route_select_knobs.argtypes = [C.c_int32, C.c_uint64]
+    lib.stc_test_route_select_knobs(first_pass, 0)
+
+
+@pytest.mark.parametrize("knob", [0, 7])
 @pytest.mark.parametrize("seed", [11, 12, 13])
-def test_random_cases_match_the_checker(seed):
+def test_random_cases_match_the_checker(seed, knob):
+    knobs(knob)
+    try:
+        run_cases(seed)
+    finally:
+        knobs(0)
+
+
+def run_cases(seed):
     rnd = random.Random(seed)
     compared = 0
     for case in range(16):
